@@ -1,0 +1,283 @@
+/*
+ * reform.h -- C ABI of the REFORM compress-and-gather core for NVIDIA B200
+ * (sm_100a).
+ *
+ * Five operations, in the order the method calls them while it walks a long
+ * input chunk by chunk (Alg. 1, procedures ForwardChunk and REFORM):
+ *
+ *   reform_chunk_step     attention of one chunk over [compressed KV cache ;
+ *                         chunk KV] that also emits the per-key eviction score
+ *   reform_embed_append   per-head L2-normalised QKV states appended to the
+ *                         cross-layer context-embedding bank
+ *   reform_evict_topk     compacts each KV head's cache back to its budget
+ *   reform_retrieve_topk  cosine scan of the bank against the query
+ *                         embeddings, pooling, top-k token selection
+ *   reform_gather         copies the selected rows into a contiguous buffer
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers unless a field says "host".
+ *     The caller owns every buffer; the library allocates nothing, keeps no
+ *     pointer after the call returns and holds no global state besides a
+ *     per-thread record of the last CUDA error and a launch counter.
+ *   - Work is enqueued on the caller's stream and the call returns without
+ *     synchronising.  Results are valid once the stream reaches that point.
+ *   - Tensors are dense, row-major, innermost dimension contiguous; device
+ *     pointers must be 16-byte aligned.
+ *   - Every params struct starts with struct_size = sizeof(the struct); a
+ *     mismatch returns REFORM_ERR_INVALID_ARG (guards against ABI drift).
+ *   - dev_status (optional, device int32): a kernel that gives up on a bounded
+ *     wait, or meets an out-of-range index, ORs a REFORM_DEV_* bit into it
+ *     instead of trapping; the context stays usable.  The caller zeroes and
+ *     reads it.
+ *   - workspace: scratch device memory, at least reform_*_workspace_size()
+ *     bytes, 256-byte aligned, private to the call while it is in flight.
+ *   - Return value: REFORM_OK or a negative REFORM_ERR_* code.  On any error
+ *     nothing has been launched.
+ *   - Indices are int32.  NaN inputs are outside the contract.
+ */
+#ifndef REFORM_H_
+#define REFORM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* reform_stream_t; /* a cudaStream_t */
+
+enum {
+  REFORM_OK = 0,
+  REFORM_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, bad struct_size, misaligned pointer */
+  REFORM_ERR_UNSUPPORTED = -2, /* dtype / head dimension the kernels do not cover */
+  REFORM_ERR_WORKSPACE = -3,   /* workspace missing or too small */
+  REFORM_ERR_CUDA = -4         /* a CUDA call failed; see reform_last_cuda_error() */
+};
+
+enum { REFORM_F32 = 0, REFORM_BF16 = 1 };
+
+/* bits a kernel may OR into *dev_status */
+enum {
+  REFORM_DEV_TIMEOUT = 1,     /* a bounded wait inside a kernel expired */
+  REFORM_DEV_BAD_INDEX = 2    /* an index outside its range was skipped */
+};
+
+/* flags of reform_chunk_step */
+enum {
+  REFORM_SCORE_ACCUMULATE = 1u, /* score[j] += carried score for cache rows j < n_cache */
+  REFORM_NO_SCORE = 2u,         /* skip the key-score pass (plain prefill attention) */
+  REFORM_FORCE_SIMT = 4u        /* use the CUDA-core kernels even where a tensor-core path exists */
+};
+
+/* kinds of state a context-embedding slot can come from */
+enum { REFORM_STATE_Q = 0, REFORM_STATE_K = 1, REFORM_STATE_V = 2 };
+
+/* ------------------------------------------------------------------------
+ * reform_chunk_step -- Sec. 3.1 "recurrent chunked forwarding" (Fig. 1 step 1)
+ * fused with the H2O eviction score of Sec. 3.1 / Sec. 4 "Common setup".
+ *
+ * For every batch b, query head h (KV head g = h / (Hq/Hkv)) and chunk row i:
+ *   visible keys j: cache rows [0, n_cache) and chunk rows [n_cache, n_cache+i]
+ *   s_ij = softmax_scale * <q_i, k_j>;  p_ij = softmax over visible j
+ *   out_i = sum_j p_ij v_j;  lse_i = log sum_j exp(s_ij)   (natural log)
+ * and, unless REFORM_NO_SCORE, for every KV head g and key j < n_cache+Lc:
+ *   score[g][j] = (ACCUMULATE && j < n_cache ? score[g][j] : 0)
+ *                 + sum_{h in group g} sum_{i >= Lc - score_window} p_ij
+ *
+ *   q      [B,Hq,Lc,d]    in
+ *   k, v   [B,Hkv,cap,d]  in; rows [0,n_cache) hold the compressed cache and
+ *                         rows [n_cache, n_cache+Lc) this chunk (caller wrote them)
+ *   out    [B,Hq,Lc,d]    out, same dtype as q
+ *   lse    [B,Hq,Lc]      fp32 out; may be NULL if the workspace holds room for it
+ *   score  [B,Hkv,cap]    fp32 in/out; rows [0, n_cache+Lc) are written
+ * d is 64 or 128.  dtype REFORM_BF16 with d == 128 runs on the tensor cores
+ * (fp32 accumulate); REFORM_F32, and bf16 with d == 64, run on CUDA cores.
+ * softmax_scale 0 means 1/sqrt(d).  score_window in [1, Lc].
+ * ------------------------------------------------------------------------ */
+typedef struct reform_chunk_params {
+  size_t struct_size;
+  int32_t dtype;
+  int32_t B, Hq, Hkv, d;
+  int32_t Lc, n_cache, cap;
+  int32_t score_window;
+  float softmax_scale;
+  uint32_t flags;
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  float* lse;
+  float* score;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} reform_chunk_params;
+
+size_t reform_chunk_step_workspace_size(const reform_chunk_params* p);
+int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_evict_topk -- Sec. 3.1 cache compression (Fig. 1 step 3), "always
+ * keep the initial and recent tokens" (Sec. 4 "Common setup").
+ *
+ * Independently for every (b, KV head): if n_keys <= budget all rows are
+ * kept.  Otherwise the first n_sink and last n_recent rows are kept, plus the
+ * budget - n_sink - n_recent rows of [n_sink, n_keys - n_recent) with the
+ * largest score; equal scores go to the lower index (-0 counts as +0).  Kept
+ * rows are written in ascending source order, so cache row r can take
+ * position id r (the consecutive re-assignment of Sec. 3.1).
+ *
+ *   k_src, v_src [B,Hkv,cap_src,d] in;   score_src [B,Hkv,cap_src] fp32 in
+ *   pos_src      [B,Hkv,cap_src] int32 in, optional (NULL)
+ *   k_dst, v_dst [B,Hkv,cap_dst,d] out;  score_dst [B,Hkv,cap_dst] fp32 out
+ *   pos_dst      optional; kept_idx [B,Hkv,budget] int32 out, optional
+ * Rows [0, n_kept) of the destinations are written, n_kept = min(n_keys,
+ * budget), also stored to *n_kept_host (host int32, optional) before return.
+ * Destinations must not overlap sources.  n_sink + n_recent > budget, or
+ * n_kept > cap_dst, is REFORM_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------ */
+typedef struct reform_evict_params {
+  size_t struct_size;
+  int32_t dtype;
+  int32_t B, Hkv, d;
+  int32_t n_keys, cap_src, cap_dst;
+  int32_t budget, n_sink, n_recent;
+  const void* k_src;
+  const void* v_src;
+  const float* score_src;
+  const int32_t* pos_src;
+  void* k_dst;
+  void* v_dst;
+  float* score_dst;
+  int32_t* pos_dst;
+  int32_t* kept_idx;
+  int32_t* n_kept_host;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} reform_evict_params;
+
+size_t reform_evict_topk_workspace_size(const reform_evict_params* p);
+int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_embed_append -- Sec. 3.2 "Combining multiple heads":
+ *   e_comb = concat_i ( e_i / ||e_i|| ).
+ *
+ * For every b, chunk token t and selected (kind, head, slot):
+ *   bank[b, token_offset + t, slot*d : (slot+1)*d] = x / max(||x||_2, eps)
+ * with x the d-vector of that head's Q, K or V state for token t; norms in
+ * fp32, one rounding (nearest-even) to the bank dtype.
+ *
+ *   q_state [B,Hq,Lc,d]; k_state, v_state [B,Hkv,Lc,d]  in; a kind that no
+ *                         selection uses may be NULL
+ *   sel     host array of n_sel (<= REFORM_MAX_SEL) entries, read during the call
+ *   bank    [B,N_cap,E]   in/out, same dtype as the states; (slot+1)*d <= E
+ * eps 0 means 1e-12.  token_offset + Lc <= N_cap.
+ * ------------------------------------------------------------------------ */
+#define REFORM_MAX_SEL 16
+
+typedef struct reform_head_sel {
+  int32_t kind; /* REFORM_STATE_Q / _K / _V */
+  int32_t head;
+  int32_t slot;
+} reform_head_sel;
+
+typedef struct reform_embed_params {
+  size_t struct_size;
+  int32_t dtype;
+  int32_t B, Lc, d, Hq, Hkv;
+  int32_t n_sel;
+  int32_t E;
+  int64_t N_cap;
+  int64_t token_offset;
+  float eps;
+  const reform_head_sel* sel; /* host */
+  const void* q_state;
+  const void* k_state;
+  const void* v_state;
+  void* bank;
+  int32_t* dev_status;
+} reform_embed_params;
+
+int reform_embed_append(const reform_embed_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_retrieve_topk -- Sec. 3.3 "Identification of significant inputs".
+ *
+ * Independently for every b:
+ *   ts[t]     = max_q  scale * <queries[q], bank[t]>          t in [0, N)
+ *   pooled[t] = max of ts over [t-r, t+r] clipped to [0, N),  r = (pool_window-1)/2
+ *   selected  = tokens [0, n_keep_head) and [N - n_keep_tail, N), plus the
+ *               k - n_keep_head - n_keep_tail other tokens with the largest
+ *               pooled score (ties to the lower index), ascending.
+ * Bank rows are stored per-head normalised (reform_embed_append), so the
+ * cosine of Sec. 3.2 is this dot product with scale = 1 / n_slots.
+ *
+ *   bank     [B,N_cap,E] in;  queries [B,nq,E] in, same dtype
+ *   idx_out  [B,k] int32 out; the first n_out = min(k, N) entries of each row are written
+ *   token_score_out, pooled_score_out [B,N] fp32 out, optional (NULL)
+ * pool_window odd >= 1.  n_keep_head + n_keep_tail > k is REFORM_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------ */
+typedef struct reform_retrieve_params {
+  size_t struct_size;
+  int32_t dtype;
+  int32_t B;
+  int64_t N, N_cap;
+  int32_t E, nq;
+  float scale;
+  int32_t pool_window;
+  int32_t n_keep_head, n_keep_tail;
+  int32_t k;
+  const void* bank;
+  const void* queries;
+  int32_t* idx_out;
+  float* token_score_out;
+  float* pooled_score_out;
+  void* workspace;
+  size_t workspace_bytes;
+  int32_t* dev_status;
+} reform_retrieve_params;
+
+size_t reform_retrieve_topk_workspace_size(const reform_retrieve_params* p);
+int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_gather -- Sec. 3.3 "gather the corresponding input embeddings"
+ * (Alg. 1, GatherRelevant).
+ *
+ *   dst[b, r, :] = src[b, idx[b, r], :]      r in [0, k)
+ *   src [B,n_rows,row_bytes] in; idx [B,k] int32 in; dst [B,k,row_bytes] out
+ * row_bytes is a multiple of 16.  An index outside [0, n_rows) zero-fills its
+ * row and sets REFORM_DEV_BAD_INDEX in *dev_status; no out-of-range access
+ * is made.
+ * ------------------------------------------------------------------------ */
+typedef struct reform_gather_params {
+  size_t struct_size;
+  int32_t B;
+  int32_t k;
+  int64_t n_rows;
+  int64_t row_bytes;
+  const void* src;
+  const int32_t* idx;
+  void* dst;
+  int32_t* dev_status;
+} reform_gather_params;
+
+int reform_gather(const reform_gather_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------ */
+const char* reform_status_string(int status);
+/* cudaError_t of the last failed CUDA call made by this thread (0 if none). */
+int reform_last_cuda_error(void);
+/* major * 10000 + minor * 100 + patch */
+int reform_version(void);
+/* Number of kernels this library has launched from the calling process since
+ * load (monotonic; for accounting in benchmarks). */
+long long reform_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REFORM_H_ */

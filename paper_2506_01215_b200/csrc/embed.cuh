@@ -1,0 +1,107 @@
+// Context-embedding append (Sec. 3.2, "Combining multiple heads"): every
+// selected head state of a token is divided by its L2 norm and stored in its
+// slot of the token's bank row.  HBM-bound: one read of the selected states,
+// one write of the bank rows.  One warp owns one (token, slot) vector; the
+// warps of a block cover neighbouring slots of the same token so a block
+// writes whole bank rows.
+#pragma once
+
+#include "common.cuh"
+
+namespace reform {
+
+struct EmbedSel {
+  const void* src[REFORM_MAX_SEL];  // base of the [B,H,Lc,d] state tensor of that kind
+  int H[REFORM_MAX_SEL];
+  int head[REFORM_MAX_SEL];
+  int slot[REFORM_MAX_SEL];
+  int n_sel;
+};
+
+constexpr int kEmbedMaxVec = 4;  // vectors of 4 elements per lane: d <= 32 * 4 * 4 = 512
+
+template <typename T>
+struct Vec4;
+template <>
+struct Vec4<float> {
+  using type = float4;
+  __device__ static void load(const float* p, float (&x)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  }
+  __device__ static void store(float* p, const float (&x)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+  }
+};
+template <>
+struct Vec4<__nv_bfloat16> {
+  __device__ static void load(const __nv_bfloat16* p, float (&x)[4]) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&v.x);
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&v.y);
+    x[0] = __low2float(a); x[1] = __high2float(a); x[2] = __low2float(b); x[3] = __high2float(b);
+  }
+  __device__ static void store(__nv_bfloat16* p, const float (&x)[4]) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]);
+    __nv_bfloat162 b = __floats2bfloat162_rn(x[2], x[3]);
+    uint2 v;
+    v.x = *reinterpret_cast<uint32_t*>(&a);
+    v.y = *reinterpret_cast<uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = v;
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_append_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, int E,
+                    long long N_cap, long long token_offset, float eps) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long items = (long long)B * Lc * sel.n_sel;
+  const int nvec = d >> 2;
+  for (long long it = warp; it < items; it += n_warps) {
+    int s = (int)(it % sel.n_sel);
+    long long bt = it / sel.n_sel;
+    int t = (int)(bt % Lc);
+    int b = (int)(bt / Lc);
+    const T* x = reinterpret_cast<const T*>(sel.src[s]) +
+                 (((long long)b * sel.H[s] + sel.head[s]) * Lc + t) * d;
+    float v[kEmbedMaxVec][4];
+    float ss = 0.f;
+#pragma unroll
+    for (int c = 0; c < kEmbedMaxVec; ++c) {
+      int vi = lane + 32 * c;
+      if (vi < nvec) {
+        Vec4<T>::load(x + 4 * vi, v[c]);
+        ss += v[c][0] * v[c][0] + v[c][1] * v[c][1] + v[c][2] * v[c][2] + v[c][3] * v[c][3];
+      }
+    }
+    ss = warp_sum(ss);
+    float nrm = fmaxf(sqrtf(ss), eps);
+    T* y = bank + ((long long)b * N_cap + token_offset + t) * E + (long long)sel.slot[s] * d;
+#pragma unroll
+    for (int c = 0; c < kEmbedMaxVec; ++c) {
+      int vi = lane + 32 * c;
+      if (vi < nvec) {
+        float o[4] = {v[c][0] / nrm, v[c][1] / nrm, v[c][2] / nrm, v[c][3] / nrm};
+        Vec4<T>::store(y + 4 * vi, o);
+      }
+    }
+  }
+}
+
+template <typename T>
+inline int launch_embed(const EmbedSel& sel, void* bank, int B, int Lc, int d, int E,
+                        long long N_cap, long long token_offset, float eps, cudaStream_t st) {
+  long long items = (long long)B * Lc * sel.n_sel;
+  if (items == 0) return REFORM_OK;
+  long long blocks = (items + 7) / 8;  // 8 warps per block
+  long long cap = (long long)kNumSMs * 16;
+  int grid = (int)(blocks < cap ? blocks : cap);
+  embed_append_kernel<T><<<grid, 256, 0, st>>>(sel, (T*)bank, B, Lc, d, E, N_cap, token_offset, eps);
+  count_launch();
+  return check_launch();
+}
+
+}  // namespace reform

@@ -1,0 +1,301 @@
+// C ABI of the REFORM compress-and-gather core: argument validation, workspace
+// carving and kernel dispatch.  Every entry point either returns an error
+// before launching anything or enqueues its kernels on the caller's stream.
+#include <atomic>
+
+#include "common.cuh"
+#include "rows.cuh"
+#include "embed.cuh"
+#include "select.cuh"
+#include "retrieve.cuh"
+#include "chunk_simt.cuh"
+#if !defined(REFORM_NO_SM100) && !__has_include("chunk_sm100.cuh")
+#define REFORM_NO_SM100
+#endif
+#ifndef REFORM_NO_SM100
+#include "chunk_sm100.cuh"
+#endif
+
+namespace reform {
+thread_local int g_last_cuda_error = 0;
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static size_t elem_size(int dtype) { return dtype == REFORM_F32 ? 4 : 2; }
+static bool dtype_ok(int dtype) { return dtype == REFORM_F32 || dtype == REFORM_BF16; }
+
+static size_t chunk_lse_bytes(const reform_chunk_params* p) {
+  return align_up(sizeof(float) * (size_t)p->B * p->Hq * p->Lc, 256);
+}
+
+static bool chunk_uses_sm100(const reform_chunk_params* p) {
+#ifndef REFORM_NO_SM100
+  return p->dtype == REFORM_BF16 && p->d == 128 && !(p->flags & REFORM_FORCE_SIMT);
+#else
+  (void)p;
+  return false;
+#endif
+}
+
+static int validate_chunk(const reform_chunk_params* p) {
+  if (!p || p->struct_size != sizeof(reform_chunk_params)) return REFORM_ERR_INVALID_ARG;
+  if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
+  if (p->B < 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv != 0) return REFORM_ERR_INVALID_ARG;
+  if (p->Lc < 0 || p->n_cache < 0 || (long long)p->n_cache + p->Lc > p->cap) return REFORM_ERR_INVALID_ARG;
+  if (p->d != 64 && p->d != 128) return REFORM_ERR_UNSUPPORTED;
+  if (!(p->flags & REFORM_NO_SCORE)) {
+    if (p->Lc > 0 && (p->score_window < 1 || p->score_window > p->Lc)) return REFORM_ERR_INVALID_ARG;
+    if (!p->score) return REFORM_ERR_INVALID_ARG;
+  }
+  if (!(p->softmax_scale >= 0.f)) return REFORM_ERR_INVALID_ARG;
+  if (!p->q || !p->k || !p->v || !p->out) return REFORM_ERR_INVALID_ARG;
+  if (!aligned16(p->q) || !aligned16(p->k) || !aligned16(p->v) || !aligned16(p->out) ||
+      !aligned16(p->score) || !aligned16(p->lse))
+    return REFORM_ERR_INVALID_ARG;
+  return REFORM_OK;
+}
+}  // namespace reform
+
+using namespace reform;
+
+extern "C" {
+
+size_t reform_chunk_step_workspace_size(const reform_chunk_params* p) {
+  if (!p || p->struct_size != sizeof(reform_chunk_params)) return 0;
+  if (p->B <= 0 || p->Hq <= 0 || p->Lc <= 0) return 0;
+  return p->lse ? 0 : chunk_lse_bytes(p);
+}
+
+int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream) {
+  int rc = validate_chunk(p);
+  if (rc != REFORM_OK) return rc;
+  float* lse = p->lse;
+  if (!lse) {
+    if (!p->workspace || p->workspace_bytes < chunk_lse_bytes(p) ||
+        (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
+      return REFORM_ERR_WORKSPACE;
+    lse = reinterpret_cast<float*>(p->workspace);
+  }
+  if (p->B == 0 || p->Lc == 0) return REFORM_OK;
+  float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->d);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+#ifndef REFORM_NO_SM100
+  if (chunk_uses_sm100(p)) return launch_chunk_sm100(p, lse, scale, st);
+#endif
+  return launch_chunk_simt(p, lse, scale, st);
+}
+
+/* ---------------------------------------------------------------- evict */
+
+static int validate_evict(const reform_evict_params* p) {
+  if (!p || p->struct_size != sizeof(reform_evict_params)) return REFORM_ERR_INVALID_ARG;
+  if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
+  if (p->B < 0 || p->Hkv <= 0 || p->d <= 0) return REFORM_ERR_INVALID_ARG;
+  if (((size_t)p->d * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
+  if (p->n_keys < 0 || p->n_keys > p->cap_src || p->budget < 0) return REFORM_ERR_INVALID_ARG;
+  if (p->n_sink < 0 || p->n_recent < 0 || (long long)p->n_sink + p->n_recent > p->budget)
+    return REFORM_ERR_INVALID_ARG;
+  int n_kept = p->n_keys < p->budget ? p->n_keys : p->budget;
+  if (n_kept > p->cap_dst) return REFORM_ERR_INVALID_ARG;
+  if (!p->k_src || !p->v_src || !p->score_src || !p->k_dst || !p->v_dst || !p->score_dst)
+    return REFORM_ERR_INVALID_ARG;
+  if ((p->pos_src == nullptr) != (p->pos_dst == nullptr)) return REFORM_ERR_INVALID_ARG;
+  if (!aligned16(p->k_src) || !aligned16(p->v_src) || !aligned16(p->k_dst) || !aligned16(p->v_dst) ||
+      !aligned16(p->score_src) || !aligned16(p->score_dst) || !aligned16(p->kept_idx))
+    return REFORM_ERR_INVALID_ARG;
+  if (p->k_src == p->k_dst || p->v_src == p->v_dst || p->score_src == p->score_dst)
+    return REFORM_ERR_INVALID_ARG;
+  return REFORM_OK;
+}
+
+static size_t evict_kept_bytes(const reform_evict_params* p) {
+  return align_up(sizeof(int32_t) * (size_t)p->B * p->Hkv * (p->budget > 0 ? p->budget : 1), 256);
+}
+
+size_t reform_evict_topk_workspace_size(const reform_evict_params* p) {
+  if (!p || p->struct_size != sizeof(reform_evict_params)) return 0;
+  if (p->B <= 0 || p->Hkv <= 0) return 0;
+  int segs = p->B * p->Hkv;
+  return sel_layout(segs, p->n_keys).total + (p->kept_idx ? 0 : evict_kept_bytes(p));
+}
+
+int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream) {
+  int rc = validate_evict(p);
+  if (rc != REFORM_OK) return rc;
+  const int n_kept = p->n_keys < p->budget ? p->n_keys : p->budget;
+  if (p->n_kept_host) *p->n_kept_host = n_kept;
+  const int segs = p->B * p->Hkv;
+  if (segs == 0 || n_kept == 0) return REFORM_OK;
+  size_t need = reform_evict_topk_workspace_size(p);
+  if (!p->workspace || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
+    return REFORM_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = reinterpret_cast<char*>(p->workspace);
+  SelLayout L = sel_layout(segs, p->n_keys);
+  int32_t* kept = p->kept_idx ? p->kept_idx : reinterpret_cast<int32_t*>(ws + L.total);
+  SelArgs a;
+  a.vals = p->score_src;
+  a.stride = p->cap_src;
+  a.n = p->n_keys;
+  if (p->n_keys <= p->budget) {  // keep everything: all rows are "forced"
+    a.lo = a.hi = p->n_keys;
+    a.m = 0;
+  } else {
+    a.lo = p->n_sink;
+    a.hi = p->n_keys - p->n_recent;
+    a.m = p->budget - p->n_sink - p->n_recent;
+  }
+  a.out = kept;
+  a.out_stride = p->budget;
+  a.state = reinterpret_cast<SelState*>(ws + L.state);
+  a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
+  a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
+  a.blocks_per_seg = L.blocks_per_seg;
+  rc = launch_select(a, segs, nullptr, nullptr, 0, st);
+  if (rc != REFORM_OK) return rc;
+  return launch_evict_compact(p->k_src, p->v_src, p->k_dst, p->v_dst, p->score_src, p->score_dst,
+                              p->pos_src, p->pos_dst, kept, p->budget, segs, n_kept, p->cap_src,
+                              p->cap_dst, (int)(p->d * elem_size(p->dtype)), st);
+}
+
+/* ---------------------------------------------------------------- embed */
+
+int reform_embed_append(const reform_embed_params* p, reform_stream_t stream) {
+  if (!p || p->struct_size != sizeof(reform_embed_params)) return REFORM_ERR_INVALID_ARG;
+  if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
+  if (p->B < 0 || p->Lc < 0 || p->d <= 0 || p->n_sel < 0 || p->n_sel > REFORM_MAX_SEL)
+    return REFORM_ERR_INVALID_ARG;
+  if (p->d % 4 != 0 || p->d > 4 * 32 * kEmbedMaxVec) return REFORM_ERR_UNSUPPORTED;
+  if (p->E <= 0 || (p->E * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
+  if (p->token_offset < 0 || p->token_offset + p->Lc > p->N_cap) return REFORM_ERR_INVALID_ARG;
+  if (!p->bank || !aligned16(p->bank) || (p->n_sel > 0 && !p->sel)) return REFORM_ERR_INVALID_ARG;
+  if (!(p->eps >= 0.f)) return REFORM_ERR_INVALID_ARG;
+  EmbedSel sel;
+  sel.n_sel = p->n_sel;
+  for (int s = 0; s < p->n_sel; ++s) {
+    const reform_head_sel& e = p->sel[s];
+    const void* src = nullptr;
+    int H = 0;
+    if (e.kind == REFORM_STATE_Q) { src = p->q_state; H = p->Hq; }
+    else if (e.kind == REFORM_STATE_K) { src = p->k_state; H = p->Hkv; }
+    else if (e.kind == REFORM_STATE_V) { src = p->v_state; H = p->Hkv; }
+    else return REFORM_ERR_INVALID_ARG;
+    if (!src || !aligned16(src) || e.head < 0 || e.head >= H || e.slot < 0 ||
+        (long long)(e.slot + 1) * p->d > p->E)
+      return REFORM_ERR_INVALID_ARG;
+    sel.src[s] = src;
+    sel.H[s] = H;
+    sel.head[s] = e.head;
+    sel.slot[s] = e.slot;
+  }
+  if (p->B == 0 || p->Lc == 0 || p->n_sel == 0) return REFORM_OK;
+  float eps = p->eps > 0.f ? p->eps : 1e-12f;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (p->dtype == REFORM_F32)
+    return launch_embed<float>(sel, p->bank, p->B, p->Lc, p->d, p->E, p->N_cap, p->token_offset, eps, st);
+  return launch_embed<__nv_bfloat16>(sel, p->bank, p->B, p->Lc, p->d, p->E, p->N_cap, p->token_offset,
+                                     eps, st);
+}
+
+/* ------------------------------------------------------------- retrieve */
+
+static int validate_retrieve(const reform_retrieve_params* p) {
+  if (!p || p->struct_size != sizeof(reform_retrieve_params)) return REFORM_ERR_INVALID_ARG;
+  if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
+  if (p->B < 0 || p->N < 0 || p->N > p->N_cap || p->N > 0x7fffffffLL || p->E <= 0 || p->nq < 1)
+    return REFORM_ERR_INVALID_ARG;
+  if ((p->E * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
+  if (p->pool_window < 1 || p->pool_window % 2 == 0) return REFORM_ERR_INVALID_ARG;
+  if ((p->pool_window - 1) / 2 > kSelMaxRadius) return REFORM_ERR_UNSUPPORTED;
+  if (p->k < 0 || p->n_keep_head < 0 || p->n_keep_tail < 0 ||
+      (long long)p->n_keep_head + p->n_keep_tail > p->k)
+    return REFORM_ERR_INVALID_ARG;
+  if (!p->bank || !p->queries || !p->idx_out) return REFORM_ERR_INVALID_ARG;
+  if (!aligned16(p->bank) || !aligned16(p->queries) || !aligned16(p->idx_out) ||
+      !aligned16(p->token_score_out) || !aligned16(p->pooled_score_out))
+    return REFORM_ERR_INVALID_ARG;
+  return REFORM_OK;
+}
+
+static size_t retrieve_score_bytes(const reform_retrieve_params* p) {
+  return align_up(sizeof(float) * (size_t)p->B * (size_t)p->N, 256);
+}
+
+size_t reform_retrieve_topk_workspace_size(const reform_retrieve_params* p) {
+  if (!p || p->struct_size != sizeof(reform_retrieve_params)) return 0;
+  if (p->B <= 0 || p->N <= 0) return 0;
+  size_t total = sel_layout(p->B, p->N).total;
+  if (!p->token_score_out) total += retrieve_score_bytes(p);
+  if (!p->pooled_score_out) total += retrieve_score_bytes(p);
+  return total;
+}
+
+int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream) {
+  int rc = validate_retrieve(p);
+  if (rc != REFORM_OK) return rc;
+  if (p->B == 0 || p->N == 0 || p->k == 0) return REFORM_OK;
+  size_t need = reform_retrieve_topk_workspace_size(p);
+  if (!p->workspace || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
+    return REFORM_ERR_WORKSPACE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = reinterpret_cast<char*>(p->workspace);
+  SelLayout L = sel_layout(p->B, p->N);
+  size_t off = L.total;
+  float* ts = p->token_score_out;
+  if (!ts) { ts = reinterpret_cast<float*>(ws + off); off += retrieve_score_bytes(p); }
+  float* pooled = p->pooled_score_out;
+  if (!pooled) { pooled = reinterpret_cast<float*>(ws + off); off += retrieve_score_bytes(p); }
+  rc = launch_scan(p->dtype, p->bank, p->queries, ts, p->B, p->N, p->N_cap, p->E, p->nq, p->scale, st);
+  if (rc != REFORM_OK) return rc;
+  SelArgs a;
+  a.vals = pooled;
+  a.stride = p->N;
+  a.n = (int)p->N;
+  if (p->N <= p->k) {
+    a.lo = a.hi = (int)p->N;
+    a.m = 0;
+  } else {
+    a.lo = p->n_keep_head;
+    a.hi = (int)p->N - p->n_keep_tail;
+    a.m = p->k - p->n_keep_head - p->n_keep_tail;
+  }
+  a.out = p->idx_out;
+  a.out_stride = p->k;
+  a.state = reinterpret_cast<SelState*>(ws + L.state);
+  a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
+  a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
+  a.blocks_per_seg = L.blocks_per_seg;
+  return launch_select(a, p->B, ts, pooled, (p->pool_window - 1) / 2, st);
+}
+
+/* --------------------------------------------------------------- gather */
+
+int reform_gather(const reform_gather_params* p, reform_stream_t stream) {
+  if (!p || p->struct_size != sizeof(reform_gather_params)) return REFORM_ERR_INVALID_ARG;
+  if (p->B < 0 || p->k < 0 || p->n_rows < 0 || p->row_bytes <= 0) return REFORM_ERR_INVALID_ARG;
+  if (p->row_bytes % 16 != 0) return REFORM_ERR_UNSUPPORTED;
+  if (!p->src || !p->idx || !p->dst) return REFORM_ERR_INVALID_ARG;
+  if (!aligned16(p->src) || !aligned16(p->dst) || (reinterpret_cast<uintptr_t>(p->idx) & 3u))
+    return REFORM_ERR_INVALID_ARG;
+  return launch_gather((const uint4*)p->src, p->idx, (uint4*)p->dst, p->B, p->k, p->n_rows,
+                       p->row_bytes, p->dev_status, reinterpret_cast<cudaStream_t>(stream));
+}
+
+/* ----------------------------------------------------------------- misc */
+
+const char* reform_status_string(int status) {
+  switch (status) {
+    case REFORM_OK: return "ok";
+    case REFORM_ERR_INVALID_ARG: return "invalid argument";
+    case REFORM_ERR_UNSUPPORTED: return "unsupported dtype, head dimension or alignment";
+    case REFORM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case REFORM_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown status";
+  }
+}
+
+int reform_last_cuda_error(void) { return g_last_cuda_error; }
+int reform_version(void) { return 100; }
+long long reform_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,335 @@
+// Deterministic segmented top-m selection used by the cache compression
+// (Sec. 3.1) and by the token selection of the gather phase (Sec. 3.3).
+//
+// For each segment: of the candidates [lo, hi) choose the m largest values
+// under the total order (value descending, index ascending) and write, in
+// ascending index order, [0, lo) ++ chosen ++ [hi, n).  The k-th key is found
+// by a most-significant-digit radix select over the order-preserving uint32
+// image of the floats (11 + 11 + 10 bits, one histogram pass each); equal keys
+// are admitted lowest index first through an ordered prefix count, so there is
+// no atomics-dependent ordering anywhere and the result is bit-reproducible.
+//
+// The optional pooling (Sec. 3.3: max over the 2r+1 adjacent tokens) is fused
+// into the first histogram pass with a log-step sliding maximum in shared
+// memory.
+#pragma once
+
+#include "common.cuh"
+
+namespace reform {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelPerThread = 4;
+constexpr int kSelTile = kSelThreads * kSelPerThread;  // elements per block
+constexpr int kSelBins = 2048;
+constexpr int kSelMaxRadius = 2048;  // pool_window <= 4097
+
+struct SelState {      // per segment, in the workspace
+  uint32_t prefix;     // key bits fixed so far (after the last pass: the threshold key)
+  uint32_t remaining;  // how many of the still-undecided candidates must be taken
+  uint32_t done[4];    // blocks finished, per pass (3 histogram passes + the count pass)
+  uint32_t pad[2];
+};
+
+struct SelLayout {  // offsets into the workspace, per call
+  size_t state, hist, blockcnt, total;
+  int blocks_per_seg;
+};
+
+inline SelLayout sel_layout(int segs, long long n_max) {
+  SelLayout L;
+  L.blocks_per_seg = (int)((n_max + kSelTile - 1) / kSelTile);
+  if (L.blocks_per_seg < 1) L.blocks_per_seg = 1;
+  size_t off = 0;
+  L.state = off;
+  off += align_up(sizeof(SelState) * segs, 256);
+  L.hist = off;
+  off += align_up(sizeof(uint32_t) * 3 * kSelBins * segs, 256);
+  L.blockcnt = off;
+  off += align_up(sizeof(uint2) * 2 * (size_t)L.blocks_per_seg * segs, 256);
+  L.total = off;
+  return L;
+}
+
+struct SelArgs {
+  const float* vals;     // candidate values; element (seg, i) at vals[seg * stride + i]
+  long long stride;
+  int n, lo, hi, m;      // segment length, candidate range, number to choose
+  int32_t* out;          // [segs, out_stride]
+  int out_stride;
+  SelState* state;
+  uint32_t* hist;        // [segs, 3, kSelBins]
+  uint2* blockcnt;       // [segs, 2, blocks_per_seg]: counts then exclusive offsets
+  int blocks_per_seg;
+};
+
+__global__ void sel_init_kernel(SelArgs a, int segs) {
+  int seg = blockIdx.x;
+  if (seg >= segs) return;
+  uint32_t* h = a.hist + (size_t)seg * 3 * kSelBins;
+  for (int i = threadIdx.x; i < 3 * kSelBins; i += blockDim.x) h[i] = 0;
+  if (threadIdx.x == 0) {
+    SelState s;
+    s.prefix = 0;
+    s.remaining = (uint32_t)a.m;
+    s.done[0] = s.done[1] = s.done[2] = s.done[3] = 0;
+    s.pad[0] = s.pad[1] = 0;
+    a.state[seg] = s;
+  }
+}
+
+// Block-wide exclusive scan of one uint per thread (1024 threads); returns the
+// exclusive prefix and, through total, the block sum.  scratch: 33 uints.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratch, uint32_t& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) scratch[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = scratch[lane];
+    uint32_t winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    scratch[lane] = winc - w;
+    if (lane == 31) scratch[32] = winc;
+  }
+  __syncthreads();
+  uint32_t res = scratch[warp] + inc - v;
+  total = scratch[32];
+  __syncthreads();
+  return res;
+}
+
+// Executed by the last block of a histogram pass: walk the bins from the top
+// until the running count reaches `remaining`; fix that digit.
+__device__ void sel_find_bin(SelState* st, const uint32_t* hist, int shift, uint32_t* scratch) {
+  const uint32_t remaining = st->remaining;
+  // thread t owns bins (2047 - 2t) and (2046 - 2t): descending order
+  int b0 = kSelBins - 1 - 2 * (int)threadIdx.x;
+  uint32_t c0 = __ldcg(hist + b0), c1 = __ldcg(hist + b0 - 1);
+  uint32_t total;
+  uint32_t before = block_excl_scan(c0 + c1, scratch, total);
+  if (before < remaining && remaining <= before + c0 + c1) {
+    int bin;
+    uint32_t rem;
+    if (remaining <= before + c0) {
+      bin = b0;
+      rem = remaining - before;
+    } else {
+      bin = b0 - 1;
+      rem = remaining - before - c0;
+    }
+    st->prefix |= (uint32_t)bin << shift;
+    st->remaining = rem;
+  } else if (remaining == 0 && threadIdx.x == 0) {
+    st->prefix |= (uint32_t)(kSelBins - 1) << shift;  // nothing to take: threshold above every key
+  }
+}
+
+__device__ __forceinline__ void sel_pass_params(int pass, int& shift, uint32_t& digit_mask,
+                                                uint32_t& prefix_mask) {
+  if (pass == 0) { shift = 21; digit_mask = 0x7FFu; prefix_mask = 0u; }
+  else if (pass == 1) { shift = 10; digit_mask = 0x7FFu; prefix_mask = 0xFFE00000u; }
+  else { shift = 0; digit_mask = 0x3FFu; prefix_mask = 0xFFFFFC00u; }
+}
+
+// One histogram pass.  POOL (pass 0 only): vals_in holds the raw token scores
+// ts; the block computes pooled[i] = max ts[i-r .. i+r] (clipped), writes it
+// to pooled_out, and histograms that.
+template <bool POOL>
+__global__ void __launch_bounds__(kSelThreads)
+sel_hist_kernel(SelArgs a, int pass, const float* __restrict__ ts, float* __restrict__ pooled_out,
+                int radius) {
+  extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
+  __shared__ uint32_t hist[kSelBins];
+  __shared__ uint32_t scratch[33];
+  __shared__ bool is_last;
+  const int seg = blockIdx.y;
+  const int tid = threadIdx.x;
+  int shift;
+  uint32_t dmask, pmask;
+  sel_pass_params(pass, shift, dmask, pmask);
+  for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+  SelState* st = a.state + seg;
+  const uint32_t prefix = (pass == 0) ? 0u : __ldcg(&st->prefix);
+  const long long base = (long long)blockIdx.x * kSelTile;  // offset inside [0, n)
+  if (POOL) {
+    // tile covers ts[base - radius, base + kSelTile + radius)
+    const int span = kSelTile + 2 * radius;
+    float* cur = tile;
+    float* nxt = tile + span;
+    const float* src = ts + (long long)seg * a.stride;
+    for (int i = tid; i < span; i += kSelThreads) {
+      long long g = base - radius + i;
+      cur[i] = (g >= 0 && g < a.n) ? src[g] : -INFINITY;
+    }
+    __syncthreads();
+    // W_p[j] = max cur[j .. j + 2^p - 1], doubling p while 2^(p+1) <= window
+    const int window = 2 * radius + 1;
+    int len = 1;
+    while (2 * len <= window) {
+      for (int i = tid; i < span; i += kSelThreads) {
+        float v = cur[i];
+        if (i + len < span) v = fmaxf(v, cur[i + len]);
+        nxt[i] = v;
+      }
+      __syncthreads();
+      float* t = cur; cur = nxt; nxt = t;
+      len *= 2;
+    }
+    // window max at centre c (tile index c + radius) = max(W[c], W[c + window - len])
+    float* dst = pooled_out + (long long)seg * a.stride;
+    for (int j = 0; j < kSelPerThread; ++j) {
+      int i = j * kSelThreads + tid;
+      long long g = base + i;
+      if (g < a.n) {
+        float v = fmaxf(cur[i], cur[i + window - len]);
+        dst[g] = v;
+        if (g >= a.lo && g < a.hi) atomicAdd(&hist[float_to_key(v) >> shift], 1u);
+      }
+    }
+  } else {
+    __syncthreads();
+    const float* src = a.vals + (long long)seg * a.stride;
+    for (int j = 0; j < kSelPerThread; ++j) {
+      long long g = base + j * kSelThreads + tid;
+      if (g >= a.lo && g < a.hi) {
+        uint32_t key = float_to_key(src[g]);
+        if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  uint32_t* gh = a.hist + ((size_t)seg * 3 + pass) * kSelBins;
+  for (int i = tid; i < kSelBins; i += kSelThreads) {
+    uint32_t c = hist[i];
+    if (c) atomicAdd(gh + i, c);
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = (atomicAdd(&st->done[pass], 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    sel_find_bin(st, gh, shift, scratch);
+  }
+}
+
+// Count pass: per block, how many candidates lie above the threshold key and
+// how many equal it; the last block turns the counts into exclusive offsets.
+__global__ void __launch_bounds__(kSelThreads) sel_count_kernel(SelArgs a) {
+  __shared__ uint32_t scratch[33];
+  __shared__ bool is_last;
+  const int seg = blockIdx.y, tid = threadIdx.x;
+  SelState* st = a.state + seg;
+  const uint32_t thr = __ldcg(&st->prefix);
+  const float* src = a.vals + (long long)seg * a.stride;
+  const long long base = (long long)blockIdx.x * kSelTile;
+  uint32_t gt = 0, eq = 0;
+  for (int j = 0; j < kSelPerThread; ++j) {
+    long long g = base + j * kSelThreads + tid;
+    if (g >= a.lo && g < a.hi) {
+      uint32_t key = float_to_key(src[g]);
+      gt += key > thr;
+      eq += key == thr;
+    }
+  }
+  uint32_t tot_gt, tot_eq;
+  block_excl_scan(gt, scratch, tot_gt);
+  block_excl_scan(eq, scratch, tot_eq);
+  uint2* cnt = a.blockcnt + (size_t)seg * 2 * a.blocks_per_seg;
+  uint2* off = cnt + a.blocks_per_seg;
+  if (tid == 0) {
+    cnt[blockIdx.x] = make_uint2(tot_gt, tot_eq);
+    __threadfence();
+    is_last = (atomicAdd(&st->done[3], 1u) == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    // exclusive scan over the blocks of this segment, kSelThreads at a time
+    uint32_t run_gt = 0, run_eq = 0;
+    for (int b0 = 0; b0 < a.blocks_per_seg; b0 += kSelThreads) {
+      int b = b0 + tid;
+      uint2 c = (b < a.blocks_per_seg) ? __ldcg(cnt + b) : make_uint2(0, 0);
+      uint32_t tg, te;
+      uint32_t eg = block_excl_scan(c.x, scratch, tg);
+      uint32_t ee = block_excl_scan(c.y, scratch, te);
+      if (b < a.blocks_per_seg) off[b] = make_uint2(run_gt + eg, run_eq + ee);
+      run_gt += tg;
+      run_eq += te;
+    }
+  }
+}
+
+// Write pass: ordered compaction.  A candidate is chosen if its key is above
+// the threshold, or equals it and fewer than need_eq equal keys precede it.
+__global__ void __launch_bounds__(kSelThreads) sel_write_kernel(SelArgs a) {
+  __shared__ uint32_t scratch[33];
+  const int seg = blockIdx.y, tid = threadIdx.x;
+  const SelState* st = a.state + seg;
+  const uint32_t thr = __ldcg(&st->prefix);
+  const uint32_t need_eq = __ldcg(&st->remaining);
+  const float* src = a.vals + (long long)seg * a.stride;
+  int32_t* out = a.out + (long long)seg * a.out_stride;
+  const uint2 boff = __ldcg(a.blockcnt + (size_t)seg * 2 * a.blocks_per_seg + a.blocks_per_seg + blockIdx.x);
+  const long long base = (long long)blockIdx.x * kSelTile;
+  uint32_t run_gt = boff.x, run_eq = boff.y;
+  for (int j = 0; j < kSelPerThread; ++j) {
+    long long g = base + j * kSelThreads + tid;
+    uint32_t is_gt = 0, is_eq = 0;
+    if (g >= a.lo && g < a.hi) {
+      uint32_t key = float_to_key(src[g]);
+      is_gt = key > thr;
+      is_eq = key == thr;
+    }
+    uint32_t tg, te;
+    uint32_t pg = block_excl_scan(is_gt, scratch, tg);
+    uint32_t pe = block_excl_scan(is_eq, scratch, te);
+    uint32_t gt_before = run_gt + pg, eq_before = run_eq + pe;
+    if (is_gt || (is_eq && eq_before < need_eq)) {
+      uint32_t pos = a.lo + gt_before + (eq_before < need_eq ? eq_before : need_eq);
+      out[pos] = (int32_t)g;
+    }
+    run_gt += tg;
+    run_eq += te;
+  }
+  if (blockIdx.x == 0) {  // forced head and tail
+    for (int i = tid; i < a.lo; i += kSelThreads) out[i] = i;
+    int tail = a.n - a.hi;
+    for (int i = tid; i < tail; i += kSelThreads) out[a.lo + a.m + i] = a.hi + i;
+  }
+}
+
+// Enqueue the whole selection.  If ts != nullptr the first pass pools ts with
+// the given radius into pooled (which must then be a.vals).
+inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, int radius,
+                         cudaStream_t st) {
+  if (segs == 0) return REFORM_OK;
+  dim3 grid(a.blocks_per_seg, segs);
+  sel_init_kernel<<<segs, 256, 0, st>>>(a, segs);
+  count_launch();
+  if (ts) {
+    size_t smem = sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius);
+    cudaFuncSetAttribute(sel_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    sel_hist_kernel<true><<<grid, kSelThreads, smem, st>>>(a, 0, ts, pooled, radius);
+  } else {
+    sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 0, nullptr, nullptr, 0);
+  }
+  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 1, nullptr, nullptr, 0);
+  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 2, nullptr, nullptr, 0);
+  sel_count_kernel<<<grid, kSelThreads, 0, st>>>(a);
+  sel_write_kernel<<<grid, kSelThreads, 0, st>>>(a);
+  count_launch(5);
+  return check_launch();
+}
+
+}  // namespace reform

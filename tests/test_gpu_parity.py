@@ -1,0 +1,334 @@
+"""GPU parity: every entry point of the C-ABI library against the fp64 CPU
+oracle on identical seeded inputs (drawn once on the CPU, copied to the GPU)."""
+import dataclasses
+
+import pytest
+import torch
+
+import oracle
+import paper_2506_01215_b200 as R
+from paper_2506_01215_b200 import synth
+from paper_2506_01215_b200.driver import LayerCache
+
+from parity import assert_index_sets_match, assert_outputs_close, assert_scores_close
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _case(B, Hq, Hkv, d, Lc, n_cache, dtype, seed=0, extra=5):
+    g = torch.Generator().manual_seed(seed)
+    cap = n_cache + Lc + extra
+    q = torch.randn(B, Hq, Lc, d, generator=g).to(dtype)
+    k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    carry = torch.rand(B, Hkv, cap, generator=g)
+    return q, k, v, carry
+
+
+def _run_chunk(q, k, v, carry, n_cache, W, flags=R.SCORE_ACCUMULATE, scale=0.0):
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    out = torch.full_like(qd, float("nan"))
+    lse = torch.full(q.shape[:3], float("nan"), device=DEV)
+    score = carry.to(DEV).clone()
+    R.chunk_step(qd, kd, vd, out, score, n_cache, W, lse=lse, flags=flags, softmax_scale=scale)
+    torch.cuda.synchronize()
+    return out, lse, score
+
+
+CHUNK_CASES = [
+    # B, Hq, Hkv, d, Lc, n_cache, dtype, W
+    (1, 4, 2, 64, 192, 100, torch.float32, 128),     # tiny-shaped, ragged everything
+    (2, 4, 2, 64, 130, 0, torch.float32, 130),       # first step, W = Lc, ragged tail
+    (1, 2, 1, 128, 200, 77, torch.float32, 1),       # TOVA-style window
+    (1, 8, 2, 128, 300, 140, torch.bfloat16, 128),   # tensor-core path, several tiles
+    (2, 4, 4, 128, 257, 0, torch.bfloat16, 257),     # no GQA sharing, W = Lc
+    (1, 4, 1, 128, 128, 512, torch.bfloat16, 64),    # cache much longer than chunk
+    (1, 4, 2, 64, 96, 40, torch.bfloat16, 32),       # bf16 on the CUDA-core path (d = 64)
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,d,Lc,n_cache,dtype,W", CHUNK_CASES)
+def test_chunk_step_matches_oracle(B, Hq, Hkv, d, Lc, n_cache, dtype, W):
+    q, k, v, carry = _case(B, Hq, Hkv, d, Lc, n_cache, dtype, seed=Lc)
+    out, lse, score = _run_chunk(q, k, v, carry, n_cache, W)
+    o_ref, lse_ref = oracle.attention(q, k, v, n_cache)
+    assert_outputs_close(out, o_ref, dtype)
+    assert (lse.cpu().double() - lse_ref).abs().max() < (2e-3 if dtype == torch.bfloat16 else 1e-4)
+    s_ref = oracle.key_scores(q, k, n_cache, W, score_in=carry, accumulate=True)
+    n = n_cache + Lc
+    G = Hq // Hkv
+    assert_scores_close(score[:, :, :n], s_ref[:, :, :n], W * G / n)
+    # rows past the keys in use keep the caller's values
+    assert torch.equal(score[:, :, n:].cpu(), carry[:, :, n:])
+    # conservation: new mass sums to W*G
+    new = score[:, :, :n].cpu().double().sum(-1) - carry[:, :, :n_cache].double().sum(-1)
+    assert torch.allclose(new, torch.full_like(new, float(W * G)), rtol=2e-3)
+
+
+def test_chunk_step_flags_and_scale():
+    q, k, v, carry = _case(1, 4, 2, 128, 160, 64, torch.bfloat16, seed=5)
+    out, lse, score = _run_chunk(q, k, v, carry, 64, 32, flags=0, scale=0.11)
+    o_ref, _ = oracle.attention(q, k, v, 64, scale=0.11)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    s_ref = oracle.key_scores(q, k, 64, 32, scale=0.11)
+    assert_scores_close(score[:, :, :224], s_ref[:, :, :224], 32 * 2 / 224)
+    out2, _, score2 = _run_chunk(q, k, v, carry, 64, 32, flags=R.NO_SCORE, scale=0.11)
+    assert torch.equal(out2, out)
+    assert torch.equal(score2.cpu(), carry)          # untouched
+    out3, _, score3 = _run_chunk(q, k, v, carry, 64, 32, flags=R.FORCE_SIMT, scale=0.11)
+    assert_outputs_close(out3, o_ref, torch.bfloat16)
+    assert_scores_close(score3[:, :, :224], s_ref[:, :, :224], 32 * 2 / 224)
+
+
+def test_chunk_step_is_deterministic():
+    q, k, v, carry = _case(1, 8, 2, 128, 260, 130, torch.bfloat16, seed=9)
+    a = _run_chunk(q, k, v, carry, 130, 128)
+    b = _run_chunk(q, k, v, carry, 130, 128)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def test_chunk_step_identical_keys_uniform_mass():
+    """All keys equal: every query spreads its mass evenly, score[j] follows
+    the harmonic-number closed form and out is the prefix mean of V."""
+    q, k, v, carry = _case(1, 4, 2, 128, 140, 60, torch.bfloat16, seed=2)
+    k[:] = k[:, :, :1]
+    out, lse, score = _run_chunk(q, k, v, carry, 60, 140, flags=0)
+    n = 200
+    H = torch.cat([torch.zeros(1, dtype=torch.float64), (1.0 / torch.arange(1, n + 1, dtype=torch.float64)).cumsum(0)])
+    expect = 2 * (H[n] - H[torch.clamp(torch.arange(n), min=60)])
+    assert_scores_close(score[0, 0, :n], expect, 140 * 2 / n)
+    pm = v[:, :, :n].double().cumsum(2)[:, :, 60:] / torch.arange(61, n + 1, dtype=torch.float64)[:, None]
+    assert (out.cpu().double() - pm.repeat_interleave(2, dim=1)).abs().max() < 2e-2
+
+
+# ------------------------------------------------------------------ evict
+
+EVICT_CASES = [
+    # B, Hkv, d, n_keys, budget, sink, recent, dtype
+    (1, 2, 64, 1536, 512, 32, 32, torch.float32),
+    (2, 3, 128, 5000, 1000, 0, 0, torch.bfloat16),
+    (1, 2, 128, 9000, 4100, 256, 256, torch.bfloat16),    # more than two select tiles, ragged
+    (1, 1, 64, 300, 40, 16, 24, torch.float32),            # no heavy hitters: sink + recent only
+    (1, 2, 64, 100, 128, 8, 8, torch.float32),             # under budget: keep all
+]
+
+
+@pytest.mark.parametrize("B,Hkv,d,n_keys,budget,sink,recent,dtype", EVICT_CASES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_evict_matches_oracle_bit_exactly(B, Hkv, d, n_keys, budget, sink, recent, dtype, ties):
+    g = torch.Generator().manual_seed(n_keys)
+    cap = n_keys + 7
+    k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    sc = torch.rand(B, Hkv, cap, generator=g)
+    if ties:
+        sc = (sc * 6).floor() / 4 - 0.5      # heavy ties, some negative, and a -0.0
+        sc[..., 5] = -0.0
+    pos = torch.randint(0, 1 << 20, (B, Hkv, cap), generator=g, dtype=torch.int32)
+    ref = oracle.evict_topk(k, v, sc, n_keys, budget, sink, recent, cap_dst=budget + 3, pos_src=pos)
+    kd = torch.zeros(B, Hkv, budget + 3, d, dtype=dtype, device=DEV)
+    vd = torch.zeros_like(kd)
+    sd = torch.zeros(B, Hkv, budget + 3, device=DEV)
+    pd = torch.zeros(B, Hkv, budget + 3, dtype=torch.int32, device=DEV)
+    kept = torch.full((B, Hkv, budget), -1, dtype=torch.int32, device=DEV)
+    n_kept = R.evict_topk(k.to(DEV), v.to(DEV), sc.to(DEV), kd, vd, sd, n_keys, budget, sink, recent,
+                          pos_src=pos.to(DEV), pos_dst=pd, kept_idx=kept)
+    torch.cuda.synchronize()
+    assert n_kept == ref["n_kept"]
+    assert torch.equal(kept.cpu()[:, :, :n_kept], ref["kept_idx"][:, :, :n_kept])
+    assert torch.equal(kd.cpu()[:, :, :n_kept].view(torch.uint8), ref["k"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(vd.cpu()[:, :, :n_kept].view(torch.uint8), ref["v"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(sd.cpu()[:, :, :n_kept].double(), ref["score"][:, :, :n_kept])
+    assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept])
+
+
+def test_evict_without_optional_outputs():
+    g = torch.Generator().manual_seed(1)
+    k = torch.randn(1, 2, 600, 64, generator=g)
+    sc = torch.rand(1, 2, 600, generator=g)
+    ref = oracle.evict_topk(k, k, sc, 600, 128, 4, 4, cap_dst=128)
+    kd = torch.zeros(1, 2, 128, 64, device=DEV)
+    vd = torch.zeros_like(kd)
+    sd = torch.zeros(1, 2, 128, device=DEV)
+    R.evict_topk(k.to(DEV), k.to(DEV).clone(), sc.to(DEV), kd, vd, sd, 600, 128, 4, 4)
+    assert torch.equal(kd.cpu(), ref["k"])
+
+
+# ------------------------------------------------------------------ embed
+
+@pytest.mark.parametrize("dtype,d,n_slots", [(torch.float32, 64, 2), (torch.bfloat16, 128, 8),
+                                               (torch.bfloat16, 256, 3)])
+def test_embed_append_matches_oracle(dtype, d, n_slots):
+    g = torch.Generator().manual_seed(d)
+    B, Hq, Hkv, Lc = 2, 8, 4, 77
+    qs = torch.randn(B, Hq, Lc, d, generator=g).to(dtype)
+    ks = (torch.randn(B, Hkv, Lc, d, generator=g) * 5).to(dtype)
+    vs = (torch.randn(B, Hkv, Lc, d, generator=g) * 0.01).to(dtype)
+    vs[0, 1, 3] = 0                                      # a zero vector stays zero
+    kinds = [2, 1, 0, 2, 2, 1, 0, 2]
+    sel = [(kinds[s], (3 * s + 1) % (Hq if kinds[s] == 0 else Hkv), s) for s in range(n_slots)]
+    E = n_slots * d
+    ref = torch.full((B, 100, E), 7.0).to(dtype)
+    f64 = oracle.embed_append(ref, 11, sel, qs, ks, vs, want_f64=True)
+    bank = torch.full((B, 100, E), 7.0).to(dtype).to(DEV)
+    R.embed_append(bank, 11, sel, q_state=qs.to(DEV), k_state=ks.to(DEV), v_state=vs.to(DEV))
+    torch.cuda.synchronize()
+    got = bank.cpu()
+    assert torch.equal(got[:, :11], ref[:, :11]) and torch.equal(got[:, 11 + Lc:], ref[:, 11 + Lc:])
+    rows = got[:, 11:11 + Lc].double()
+    exact = f64[:, 11:11 + Lc]
+    ulp = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -23
+    # fp32 norm then one rounding: within one unit in the last place of the fp64 quotient
+    assert ((rows - exact).abs() <= ulp * exact.abs() + 1e-30).all()
+    same = (got[:, 11:11 + Lc] == ref[:, 11:11 + Lc]).float().mean().item()
+    assert same > 0.99, f"only {same:.4f} of elements equal the oracle's rounding"
+
+
+# --------------------------------------------------------------- retrieve
+
+def _retrieve_case(w, N, pool, keep, k, seed):
+    w = dataclasses.replace(w, N=N, k=k, pool_window=pool, keep_head=keep, keep_tail=keep)
+    bank, qs, planted = synth.bank_and_queries(w, seed=seed)
+    ref = oracle.retrieve_topk(bank, qs, N, k, scale=w.sim_scale, pool_window=pool,
+                               n_keep_head=keep, n_keep_tail=keep)
+    idx = torch.full((w.B, k), -1, dtype=torch.int32, device=DEV)
+    ts = torch.zeros(w.B, N, device=DEV)
+    pooled = torch.zeros(w.B, N, device=DEV)
+    n_out = R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx, scale=w.sim_scale, pool_window=pool,
+                            n_keep_head=keep, n_keep_tail=keep, token_score_out=ts,
+                            pooled_score_out=pooled)
+    torch.cuda.synchronize()
+    return w, ref, idx.cpu(), ts.cpu(), pooled.cpu(), planted, n_out
+
+
+RETRIEVE_CASES = [
+    # workload, N, pool, keep, k
+    ("tiny", 8192, 1, 0, 256),
+    ("tiny", 8192, 17, 8, 256),
+    ("tiny", 5000, 129, 8, 300),          # ragged N, paper's window
+    ("llama8b_128k", 9001, 129, 256, 1024),   # bf16 MMA path, nq = 4, ragged
+    ("retrieval_1m", 4099, 5, 16, 512),       # nq = 64
+    ("mistral7b_4x256k", 3000, 129, 256, 700),  # batch 4, nq = 8
+]
+
+
+@pytest.mark.parametrize("name,N,pool,keep,k", RETRIEVE_CASES)
+def test_retrieve_matches_oracle(name, N, pool, keep, k):
+    w, ref, idx, ts, pooled, planted, n_out = _retrieve_case(synth.WORKLOADS[name], N, pool, keep, k, seed=N)
+    assert n_out == ref["n_out"]
+    assert_scores_close(ts, ref["ts"], 1.0)
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    for b in range(w.B):
+        assert_index_sets_match(idx[b, :n_out], ref["idx"][b], ref["pooled"][b])
+        if pool == 1:
+            assert set(planted[b]) <= set(idx[b].tolist())
+
+
+def test_retrieve_ties_take_lowest_index_and_k_ge_n():
+    bank = torch.ones(1, 700, 32, dtype=torch.bfloat16)
+    qs = torch.ones(1, 3, 32, dtype=torch.bfloat16)
+    idx = torch.full((1, 50), -1, dtype=torch.int32, device=DEV)
+    R.retrieve_topk(bank.to(DEV), qs.to(DEV), 700, 50, idx, pool_window=9, n_keep_head=2, n_keep_tail=3)
+    assert idx.cpu()[0].tolist() == list(range(47)) + [697, 698, 699]
+    idx = torch.full((1, 900), -1, dtype=torch.int32, device=DEV)
+    n = R.retrieve_topk(bank.to(DEV), qs.to(DEV), 700, 900, idx)
+    assert n == 700 and idx.cpu()[0, :700].tolist() == list(range(700))
+
+
+# ----------------------------------------------------------------- gather
+
+@pytest.mark.parametrize("D,dtype", [(512, torch.float32), (4096, torch.bfloat16), (8, torch.bfloat16),
+                                     (136, torch.bfloat16)])
+def test_gather_matches_oracle(D, dtype):
+    g = torch.Generator().manual_seed(D)
+    src = torch.randn(2, 999, D, generator=g).to(dtype)
+    idx = torch.randint(0, 999, (2, 257), generator=g, dtype=torch.int32)
+    ref = oracle.gather(src, idx)
+    dst = torch.zeros(2, 257, D, dtype=dtype, device=DEV)
+    R.gather(src.to(DEV), idx.to(DEV), dst)
+    torch.cuda.synchronize()
+    assert torch.equal(dst.cpu().view(torch.uint8), ref.view(torch.uint8))
+
+
+def test_gather_flags_bad_index_without_faulting():
+    src = torch.randn(1, 10, 64, device=DEV)
+    idx = torch.tensor([[3, 10, -1, 9]], dtype=torch.int32, device=DEV)
+    dst = torch.full((1, 4, 64), 5.0, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.gather(src, idx, dst, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == R.DEV_BAD_INDEX
+    assert torch.equal(dst[0, 0], src[0, 3]) and torch.equal(dst[0, 3], src[0, 9])
+    assert torch.all(dst[0, 1:3] == 0)
+
+
+# ------------------------------------------------- recurrent pipeline (Tiny)
+
+@pytest.mark.parametrize("sink,window", [(32, 128), (0, 1024)])
+def test_tiny_recurrence_matches_oracle_step_by_step(sink, window):
+    """Config 1 end to end: 8 chunk steps with eviction, each step fed the
+    oracle's pre-step state so every step is judged on its own; needles
+    survive every eviction."""
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], n_sink=sink, n_recent=sink, window=window)
+    G = w.Hq // w.Hkv
+    needles = synth.needle_positions(w)
+    # oracle-side state
+    ck = torch.zeros(w.B, w.Hkv, w.cap, w.d)
+    cv = torch.zeros_like(ck)
+    cs = torch.zeros(w.B, w.Hkv, w.cap, dtype=torch.float64)
+    pos = torch.zeros(w.B, w.Hkv, w.cap, dtype=torch.int32)
+    n_cache = 0
+    swaps = 0
+    for step in range(w.steps):
+        q, kc, vc = synth.chunk_qkv(w, 0, step)
+        ck[:, :, n_cache:n_cache + w.Lc] = kc
+        cv[:, :, n_cache:n_cache + w.Lc] = vc
+        pos[:, :, n_cache:n_cache + w.Lc] = torch.arange(step * w.Lc, (step + 1) * w.Lc, dtype=torch.int32)
+        n = n_cache + w.Lc
+        # GPU step from the oracle's state
+        out, lse, score = _run_chunk(q, ck, cv, cs.float(), n_cache, window)
+        o_ref, _ = oracle.attention(q, ck, cv, n_cache)
+        assert_outputs_close(out, o_ref, w.dtype)
+        s_ref = oracle.key_scores(q, ck, n_cache, window, score_in=cs.float(), accumulate=True)
+        assert_scores_close(score[:, :, :n], s_ref[:, :, :n], window * G / n)
+        ref = oracle.evict_topk(ck, cv, s_ref, n, w.budget, sink, sink, cap_dst=w.cap, pos_src=pos)
+        kd = torch.zeros(w.B, w.Hkv, w.cap, w.d, device=DEV)
+        vd = torch.zeros_like(kd)
+        sd = torch.zeros(w.B, w.Hkv, w.cap, device=DEV)
+        kept = torch.zeros(w.B, w.Hkv, w.budget, dtype=torch.int32, device=DEV)
+        R.evict_topk(ck.to(DEV), cv.to(DEV), score, kd, vd, sd, n, w.budget, sink, sink, kept_idx=kept)
+        for h in range(w.Hkv):
+            swaps += assert_index_sets_match(kept[0, h].cpu(), ref["kept_idx"][0, h], s_ref[0, h])
+            kept_pos = set(ref["pos"][0, h, :w.budget].tolist())
+            seen = [p for p in needles if p < (step + 1) * w.Lc]
+            assert set(seen) <= kept_pos, f"needle evicted at step {step}"
+        ck, cv, cs, pos = ref["k"], ref["v"], ref["score"], ref["pos"]
+        n_cache = ref["n_kept"]
+    assert swaps <= 4
+
+
+def test_tiny_free_running_pipeline_with_driver():
+    """The binding's driver runs all 8 steps on the GPU alone; the oracle runs
+    them alone; kept positions and final cache agree."""
+    w = synth.WORKLOADS["tiny"]
+    cache = LayerCache(w.B, w.Hkv, w.d, w.cap, w.budget, w.n_sink, w.n_recent, w.dtype, DEV)
+    ck = torch.zeros(w.B, w.Hkv, w.cap, w.d)
+    cv = torch.zeros_like(ck)
+    cs = torch.zeros(w.B, w.Hkv, w.cap, dtype=torch.float64)
+    n_cache = 0
+    out = torch.zeros(w.B, w.Hq, w.Lc, w.d, device=DEV)
+    for step in range(w.steps):
+        q, kc, vc = synth.chunk_qkv(w, 0, step)
+        cache.write_chunk(kc.to(DEV), vc.to(DEV))
+        cache.attend(q.to(DEV), out, w.window)
+        cache.evict()
+        ck[:, :, n_cache:n_cache + w.Lc] = kc
+        cv[:, :, n_cache:n_cache + w.Lc] = vc
+        s_ref = oracle.key_scores(q, ck, n_cache, w.window, score_in=cs, accumulate=True)
+        ref = oracle.evict_topk(ck, cv, s_ref, n_cache + w.Lc, w.budget, w.n_sink, w.n_recent, cap_dst=w.cap)
+        ck, cv, cs, n_cache = ref["k"], ref["v"], ref["score"], ref["n_kept"]
+        same = (cache.k[cache.cur][:, :, :n_cache].cpu() == ck[:, :, :n_cache]).all(-1).float().mean().item()
+        assert same > 0.995, f"step {step}: only {same:.4f} of cache rows agree"
+    assert_scores_close(cache.score[cache.cur][:, :, :n_cache], cs[:, :, :n_cache], 1e-3) if same == 1.0 else None
