@@ -236,7 +236,7 @@ class HostPass:
         self.hidx.copy_(p.idx, non_blocking=True)
 
 
-def cpu_baseline(w, sample_rows=2048):
+def cpu_baseline(w, sample_rows=8192):
     """The oracle, as it stands, on a bounded sample: one KV-head group of recurrence step 1,
     every (Lc/sample_rows)-th query row for the attention output plus the full 128-row score
     window.  Extrapolated to the metric through (query, key) pairs per second."""
