@@ -1,0 +1,463 @@
+// Tensor-core chunk step for bf16, head dimension 128 (sm_100a: tcgen05 MMA
+// with TMEM accumulators, operands staged by TMA with 128-byte swizzle).
+//
+//   attn_sm100_kernel   Sec. 3.1 chunk forward.  One block owns a 128-row query
+//     tile of one head and walks the visible keys [cache ; chunk prefix] in
+//     128-key tiles:  S = Q K^T (SS MMA, fp32 in TMEM) -> online softmax by 128
+//     threads, one query row each, straight out of TMEM -> P (bf16) written
+//     back into the TMEM columns S occupied -> O += P V (A operand from TMEM, V
+//     from shared memory, MN-major).  O stays in TMEM for the whole walk and is
+//     rescaled only when a row maximum grows by more than 2^8.  Two blocks are
+//     resident per SM (256 TMEM columns, 96 KB of shared memory each): while
+//     one block's softmax runs, the other block's MMAs keep the tensor pipe busy.
+//
+//   score_sm100_kernel  H2O eviction score (Sec. 3.1; Sec. 4 "Common setup").
+//     Key-stationary second pass: a block owns 128 keys (TMEM lanes) of one KV
+//     head and revisits the trailing score_window query rows of the group's G
+//     query heads: S^T = K Q^T, p = exp2(s*c - lse), summed along the queries
+//     by the thread that owns the key.  One owner per key: no atomics, and the
+//     result does not depend on scheduling.
+//
+// Roles per block (192 threads): warp 0 = TMA producer (one lane), warp 1 =
+// MMA issuer (one lane) and TMEM owner, warps 2..5 = 128 softmax/epilogue
+// threads (TMEM lane = 32 * (warp % 4) + lane).  All waits are bounded.
+#pragma once
+
+#include "common.cuh"
+#include "chunk_simt.cuh"
+#include "sm100_ptx.cuh"
+
+namespace reform {
+
+constexpr int kT = 128;                   // tile edge: query rows, keys, head dimension
+constexpr int kSm100Threads = 192;
+constexpr uint32_t kTileBytes = kT * kT * 2;  // one 128 x 128 bf16 tile
+constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one TMA box: 128 rows x 64 columns
+constexpr uint32_t kTmemCols = 256;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+constexpr size_t kAttnSmemBytes = 3 * kTileBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr size_t kScoreSmemBytes = 3 * kTileBytes + 1024 + 256 + 2 * kT * sizeof(float);
+
+__device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
+  return reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(p) + 1023) & ~uintptr_t(1023));
+}
+
+// S (or S^T) = A B^T for two K-major 128 x 128 bf16 tiles in shared memory: 8 MMAs of K = 16
+__device__ __forceinline__ void issue_kmajor_128x128x128(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
+  constexpr uint32_t idesc = ptx::idesc_bf16(kT, kT, false, false);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;  // 64-column box, then 32 B per K = 16 step
+    ptx::mma_ss(d_tmem, ptx::smem_desc_sw128(a_smem + off, 16, 1024),
+                ptx::smem_desc_sw128(b_smem + off, 16, 1024), idesc, k > 0);
+  }
+}
+
+__global__ void __launch_bounds__(kSm100Threads, 2)
+attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ out,
+                  float* __restrict__ lse, int Hq, int Hkv, int Lc, int n_cache, float scale_log2,
+                  int32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align_1024(smem_raw);
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + kTileBytes;
+  uint8_t* sV = smem + 2 * kTileBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 3 * kTileBytes);
+  uint64_t* q_full = bars + 0;
+  uint64_t* k_full = bars + 1;
+  uint64_t* k_empty = bars + 2;
+  uint64_t* v_full = bars + 3;
+  uint64_t* v_empty = bars + 4;
+  uint64_t* s_full = bars + 5;
+  uint64_t* p_ready = bars + 6;
+  uint64_t* o_full = bars + 7;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_qt = (Lc + kT - 1) / kT;
+  const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
+  const int h = blockIdx.y % Hq, b = blockIdx.y / Hq;
+  const int g = h / (Hq / Hkv);
+  const int row0 = qt * kT;
+  const int last_row = min(row0 + kT - 1, Lc - 1);
+  const int n_kt = (n_cache + last_row + 1 + kT - 1) / kT;  // key tiles with at least one visible key
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(q_full, 1);
+    ptx::mbar_init(k_full, 1);
+    ptx::mbar_init(k_empty, 1);
+    ptx::mbar_init(v_full, 1);
+    ptx::mbar_init(v_empty, 1);
+    ptx::mbar_init(s_full, 1);
+    ptx::mbar_init(p_ready, 128);
+    ptx::mbar_init(o_full, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tS = tmem_base;        // columns [0, 128): S (fp32), later P (bf16, columns [0, 64))
+  const uint32_t tO = tmem_base + kT;   // columns [128, 256): O (fp32)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::prefetch_tmap(&tmQ);
+      ptx::prefetch_tmap(&tmK);
+      ptx::prefetch_tmap(&tmV);
+      ptx::mbar_expect_tx(q_full, kTileBytes);
+      ptx::tma_load_3d(sQ, &tmQ, q_full, 0, row0, b * Hq + h);
+      ptx::tma_load_3d(sQ + kHalfBytes, &tmQ, q_full, 64, row0, b * Hq + h);
+      int issued_k = 0, issued_v = 0;
+      for (int j = 0; j < n_kt; ++j) {
+        if (!ptx::mbar_wait(k_empty, (j & 1) ^ 1, abort_flag)) break;
+        ptx::mbar_expect_tx(k_full, kTileBytes);
+        ptx::tma_load_3d(sK, &tmK, k_full, 0, j * kT, b * Hkv + g);
+        ptx::tma_load_3d(sK + kHalfBytes, &tmK, k_full, 64, j * kT, b * Hkv + g);
+        issued_k = j + 1;
+        if (!ptx::mbar_wait(v_empty, (j & 1) ^ 1, abort_flag)) break;
+        ptx::mbar_expect_tx(v_full, kTileBytes);
+        ptx::tma_load_3d(sV, &tmV, v_full, 0, j * kT, b * Hkv + g);
+        ptx::tma_load_3d(sV + kHalfBytes, &tmV, v_full, 64, j * kT, b * Hkv + g);
+        issued_v = j + 1;
+      }
+      if (*abort_flag) {  // let copies in flight land before the block's shared memory is released
+        volatile int ignore = 0;
+        ptx::mbar_wait(q_full, 0, &ignore);
+        if (issued_k) ptx::mbar_wait(k_full, (issued_k - 1) & 1, &ignore);
+        if (issued_v) ptx::mbar_wait(v_full, (issued_v - 1) & 1, &ignore);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = ptx::idesc_bf16(kT, kT, false, true);  // V is MN-major
+      const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK), aV = ptx::smem_u32(sV);
+      bool ok = ptx::mbar_wait(q_full, 0, abort_flag);
+      for (int j = 0; ok && j < n_kt; ++j) {
+        if (!ptx::mbar_wait(k_full, j & 1, abort_flag)) break;
+        ptx::tc_fence_after();
+        issue_kmajor_128x128x128(tS, aQ, aK);
+        ptx::mma_commit(s_full);
+        ptx::mma_commit(k_empty);
+        if (!ptx::mbar_wait(p_ready, j & 1, abort_flag)) break;
+        if (!ptx::mbar_wait(v_full, j & 1, abort_flag)) break;
+        ptx::tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          // A: P columns [8k, 8k+8) = keys [16k, 16k+16); B: V rows [16k, 16k+16), both 64-column halves
+          ptx::mma_ts(tO, tS + 8 * k, ptx::smem_desc_sw128(aV + k * 2048, kHalfBytes, 1024), idesc_pv,
+                      (j > 0) || (k > 0));
+        }
+        ptx::mma_commit(v_empty);
+        if (j == n_kt - 1) ptx::mma_commit(o_full);
+      }
+    }
+  } else {
+    const int sub = warp & 3;                     // TMEM sub-partition of this warp
+    const int r = 32 * sub + lane;                // row of the tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)(32 * sub) << 16;
+    const int row = row0 + r;
+    const int lim = n_cache + row;                // last visible key of this row
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kt; ++j) {
+      if (!ptx::mbar_wait(s_full, j & 1, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const int key0 = j * kT;
+      const bool need_mask = key0 + kT - 1 > n_cache + row0;
+      uint32_t v[32];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        ptx::tmem_ld32(tS + lane_addr + 32 * c, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float x = __uint_as_float(v[i]);
+          if (need_mask && key0 + 32 * c + i > lim) x = -INFINITY;
+          mx = fmaxf(mx, x);
+        }
+      }
+      const float m_new = fmaxf(m, mx * scale_log2);
+      if (j == 0) {
+        m = m_new;  // key 0 is visible to every row, so m is finite from here on
+      } else {
+        const bool grow = m_new > m + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
+          if (grow) m = m_new;
+          l *= alpha;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            ptx::tmem_ld32(tO + lane_addr + 32 * c, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+            ptx::tmem_st32(tO + lane_addr + 32 * c, v);
+          }
+          ptx::tmem_st_wait();
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        ptx::tmem_ld32(tS + lane_addr + 32 * c, v);
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          float p0 = ptx::ex2(fmaf(__uint_as_float(v[i]), scale_log2, -m));
+          float p1 = ptx::ex2(fmaf(__uint_as_float(v[i + 1]), scale_log2, -m));
+          if (need_mask) {
+            if (key0 + 32 * c + i > lim) p0 = 0.f;
+            if (key0 + 32 * c + i + 1 > lim) p1 = 0.f;
+          }
+          l += p0 + p1;
+          pk[i >> 1] = ptx::pack_bf16(p0, p1);
+        }
+        ptx::tmem_st16(tS + lane_addr + 16 * c, pk);
+      }
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(p_ready);
+    }
+    if (ok && ptx::mbar_wait(o_full, 0, abort_flag)) {
+      ptx::tc_fence_after();
+      const float inv = 1.0f / l;
+      __nv_bfloat16* op = out + (((long long)b * Hq + h) * Lc + row) * kT;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        ptx::tmem_ld32(tO + lane_addr + 32 * c, v);
+        if (row < Lc) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 o;
+            o.x = ptx::pack_bf16(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
+            o.y = ptx::pack_bf16(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+            o.z = ptx::pack_bf16(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
+            o.w = ptx::pack_bf16(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(op + 32 * c + i) = o;
+          }
+        }
+      }
+      if (row < Lc) lse[((long long)b * Hq + h) * Lc + row] = (m + log2f(l)) * kLn2;
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+}
+
+// Enumerates the (query head of the group, 128-row query tile of the window)
+// pairs a key tile has to visit, skipping tiles none of whose rows sees it.
+struct ScoreTiles {
+  int G, Lc, n_cache, i_begin, j0;
+  int hh, i0;
+  __device__ ScoreTiles(int G_, int Lc_, int n_cache_, int window, int j0_)
+      : G(G_), Lc(Lc_), n_cache(n_cache_), i_begin(Lc_ - window), j0(j0_), hh(0), i0(Lc_ - window) {
+    skip();
+  }
+  __device__ bool valid() const { return hh < G; }
+  __device__ void next() {
+    i0 += kT;
+    if (i0 >= Lc) { i0 = i_begin; ++hh; }
+    skip();
+  }
+  __device__ void skip() {
+    while (hh < G && j0 > n_cache + min(i0 + kT - 1, Lc - 1)) {
+      i0 += kT;
+      if (i0 >= Lc) { i0 = i_begin; ++hh; }
+    }
+  }
+};
+
+__global__ void __launch_bounds__(kSm100Threads, 2)
+score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const float* __restrict__ lse, float* __restrict__ score, int Hq, int Hkv, int Lc,
+                   int n_cache, int cap, int window, float scale_log2, int accumulate,
+                   int32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align_1024(smem_raw);
+  uint8_t* sK = smem;
+  uint8_t* sQ = smem + kTileBytes;  // two stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 3 * kTileBytes);
+  uint64_t* k_full = bars + 0;
+  uint64_t* q_full = bars + 1;   // [2]
+  uint64_t* q_empty = bars + 3;  // [2]
+  uint64_t* d_full = bars + 5;   // [2]
+  uint64_t* d_empty = bars + 7;  // [2]
+  uint64_t* lse_ready = bars + 9;  // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 11);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* lse2 = reinterpret_cast<float*>(smem + 3 * kTileBytes + 256);  // [2][128]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.y % Hkv, b = blockIdx.y / Hkv;
+  const int G = Hq / Hkv;
+  const int n = n_cache + Lc;
+  const int j0 = blockIdx.x * kT;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(k_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(q_full + s, 1);
+      ptx::mbar_init(q_empty + s, 1);
+      ptx::mbar_init(d_full + s, 1);
+      ptx::mbar_init(d_empty + s, 128);
+      ptx::mbar_init(lse_ready + s, 128);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      ptx::prefetch_tmap(&tmQ);
+      ptx::prefetch_tmap(&tmK);
+      ptx::mbar_expect_tx(k_full, kTileBytes);
+      ptx::tma_load_3d(sK, &tmK, k_full, 0, j0, b * Hkv + g);
+      ptx::tma_load_3d(sK + kHalfBytes, &tmK, k_full, 64, j0, b * Hkv + g);
+      int it = 0;
+      for (ScoreTiles t(G, Lc, n_cache, window, j0); t.valid(); t.next(), ++it) {
+        const int s = it & 1;
+        if (!ptx::mbar_wait(q_empty + s, ((it >> 1) & 1) ^ 1, abort_flag)) break;
+        ptx::mbar_expect_tx(q_full + s, kTileBytes);
+        uint8_t* dst = sQ + s * kTileBytes;
+        ptx::tma_load_3d(dst, &tmQ, q_full + s, 0, t.i0, b * Hq + g * G + t.hh);
+        ptx::tma_load_3d(dst + kHalfBytes, &tmQ, q_full + s, 64, t.i0, b * Hq + g * G + t.hh);
+      }
+      if (*abort_flag) {
+        volatile int ignore = 0;
+        ptx::mbar_wait(k_full, 0, &ignore);
+        for (int u = 1; u <= 2 && u <= it; ++u) {
+          int last = it - u;
+          ptx::mbar_wait(q_full + (last & 1), (last >> 1) & 1, &ignore);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t aK = ptx::smem_u32(sK), aQ = ptx::smem_u32(sQ);
+      bool ok = ptx::mbar_wait(k_full, 0, abort_flag);
+      int it = 0;
+      for (ScoreTiles t(G, Lc, n_cache, window, j0); ok && t.valid(); t.next(), ++it) {
+        const int s = it & 1, ph = (it >> 1) & 1;
+        if (!ptx::mbar_wait(q_full + s, ph, abort_flag)) break;
+        if (!ptx::mbar_wait(d_empty + s, ph ^ 1, abort_flag)) break;
+        ptx::tc_fence_after();
+        issue_kmajor_128x128x128(tmem_base + s * kT, aK, aQ + s * kTileBytes);
+        ptx::mma_commit(d_full + s);
+        ptx::mma_commit(q_empty + s);
+      }
+    }
+  } else {
+    const int sub = warp & 3;
+    const int r = 32 * sub + lane;
+    const uint32_t lane_addr = (uint32_t)(32 * sub) << 16;
+    const int key = j0 + r;
+    float acc = 0.f;
+    int it = 0;
+    for (ScoreTiles t(G, Lc, n_cache, window, j0); t.valid(); t.next(), ++it) {
+      const int s = it & 1, ph = (it >> 1) & 1;
+      const int qi = t.i0 + r;
+      lse2[s * kT + r] = (qi < Lc) ? lse[((long long)b * Hq + g * G + t.hh) * Lc + qi] * kLog2e : INFINITY;
+      ptx::mbar_arrive(lse_ready + s);
+      if (!ptx::mbar_wait(lse_ready + s, ph, abort_flag)) break;
+      if (!ptx::mbar_wait(d_full + s, ph, abort_flag)) break;
+      ptx::tc_fence_after();
+      const int vis0 = key - n_cache - t.i0;  // column c sees this key iff c >= vis0
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        ptx::tmem_ld32(tmem_base + s * kT + lane_addr + 32 * c, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float p = ptx::ex2(fmaf(__uint_as_float(v[i]), scale_log2, -lse2[s * kT + 32 * c + i]));
+          if (32 * c + i >= vis0) acc += p;
+        }
+      }
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(d_empty + s);
+    }
+    if (key < n && !*abort_flag) {
+      long long o = ((long long)b * Hkv + g) * cap + key;
+      float carry = (accumulate && key < n_cache) ? score[o] : 0.f;
+      score[o] = carry + acc;
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+}
+
+inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float scale, cudaStream_t st) {
+  const int n = p->n_cache + p->Lc;
+  const float scale_log2 = scale * kLog2e;
+  CUtensorMap tmQ, tmK, tmV;
+  if (!make_tmap_bf16_d128(&tmQ, p->q, (long long)p->B * p->Hq, p->Lc, p->Lc, kT) ||
+      !make_tmap_bf16_d128(&tmK, p->k, (long long)p->B * p->Hkv, n, p->cap, kT) ||
+      !make_tmap_bf16_d128(&tmV, p->v, (long long)p->B * p->Hkv, n, p->cap, kT)) {
+    g_last_cuda_error = (int)cudaErrorInvalidValue;
+    return REFORM_ERR_CUDA;
+  }
+  int mode = 0;  // bring-up aid: 1 = tensor-core score pass only, 2 = tensor-core attention only
+  if (const char* e = getenv("REFORM_SM100_MODE")) mode = atoi(e);
+  int rc;
+  if (mode == 1) {
+    reform_chunk_params q = *p;
+    q.flags |= REFORM_NO_SCORE;
+    rc = launch_chunk_simt(&q, lse, scale, st);
+    if (rc != REFORM_OK) return rc;
+  } else {
+    cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+    dim3 grid((p->Lc + kT - 1) / kT, p->B * p->Hq);
+    attn_sm100_kernel<<<grid, kSm100Threads, kAttnSmemBytes, st>>>(
+        tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
+        p->dev_status);
+    count_launch();
+    rc = check_launch();
+    if (rc != REFORM_OK) return rc;
+  }
+  if (p->flags & REFORM_NO_SCORE) return REFORM_OK;
+  if (mode == 2) {
+    const float sl2 = scale_log2;
+    cudaFuncSetAttribute(score_simt_kernel<__nv_bfloat16, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)SimtSmem<128>::score_bytes);
+    dim3 grid2((n + kBN - 1) / kBN, p->B * p->Hkv);
+    score_simt_kernel<__nv_bfloat16, 128><<<grid2, kSimtThreads, SimtSmem<128>::score_bytes, st>>>(
+        (const __nv_bfloat16*)p->q, (const __nv_bfloat16*)p->k, lse, p->score, p->Hq, p->Hkv, p->Lc,
+        p->n_cache, p->cap, p->score_window, sl2, (p->flags & REFORM_SCORE_ACCUMULATE) ? 1 : 0);
+    count_launch();
+    return check_launch();
+  }
+  cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScoreSmemBytes);
+  dim3 grid2((n + kT - 1) / kT, p->B * p->Hkv);
+  score_sm100_kernel<<<grid2, kSm100Threads, kScoreSmemBytes, st>>>(
+      tmQ, tmK, lse, p->score, p->Hq, p->Hkv, p->Lc, p->n_cache, p->cap, p->score_window, scale_log2,
+      (p->flags & REFORM_SCORE_ACCUMULATE) ? 1 : 0, p->dev_status);
+  count_launch();
+  return check_launch();
+}
+
+}  // namespace reform
