@@ -257,6 +257,283 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
 }
 
+
+// ---------------------------------------------------------------------------
+// Two query tiles per block, one block per SM.  The two tiles (normally the
+// same 128 query rows of two query heads of one KV group, so their walks are
+// identical) share every K/V tile a single TMA load brings in: half the
+// L2 -> shared-memory traffic per flop of a one-tile block.  Each tile has its
+// own S/P and O accumulators in tensor memory (4 x 128 = all 512 columns) and
+// its own warpgroup of 128 softmax threads holding a whole 128-wide row in
+// registers; the MMA issuer alternates between the tiles, so one tile's
+// softmax hides behind the other tile's two MMAs.
+// ---------------------------------------------------------------------------
+constexpr int kAttn2Threads = 384;  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
+constexpr size_t kAttn2SmemBytes = 6 * kTileBytes + 1024 + 512;
+
+struct Attn2Tile {
+  int head;    // b * Hq + query head, or -1 if this block has no second tile
+  int row0;    // first chunk row of the tile
+  int n_kt;    // key tiles to walk (0 if absent)
+};
+
+__device__ __forceinline__ Attn2Tile attn2_tile(int u, int U, int G, int n_qt, int bg_q0, int Lc,
+                                                int n_cache) {
+  Attn2Tile t;
+  if (u >= U) {
+    t.head = -1; t.row0 = 0; t.n_kt = 0;
+    return t;
+  }
+  const int qt = n_qt - 1 - u / G;  // longest walks first
+  t.head = bg_q0 + u % G;
+  t.row0 = qt * kT;
+  const int last_row = min(t.row0 + kT - 1, Lc - 1);
+  t.n_kt = (n_cache + last_row + 1 + kT - 1) / kT;
+  return t;
+}
+
+__global__ void __launch_bounds__(kAttn2Threads, 1)
+attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                   const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ out,
+                   float* __restrict__ lse, int Hq, int Hkv, int Lc, int n_cache, float scale_log2,
+                   int32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = align_1024(smem_raw);
+  uint8_t* sQ = smem;                    // [2] query tiles
+  uint8_t* sK = smem + 2 * kTileBytes;   // [2] stages
+  uint8_t* sV = smem + 4 * kTileBytes;   // [2] stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * kTileBytes);
+  uint64_t* q_full = bars + 0;
+  uint64_t* k_full = bars + 1;    // [2]
+  uint64_t* k_empty = bars + 3;   // [2]
+  uint64_t* v_full = bars + 5;    // [2]
+  uint64_t* v_empty = bars + 7;   // [2]
+  uint64_t* s_full = bars + 9;    // [2] per tile
+  uint64_t* p_ready = bars + 11;  // [2] per tile
+  uint64_t* o_full = bars + 13;   // [2] per tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = Hq / Hkv;
+  const int g = blockIdx.y % Hkv, b = blockIdx.y / Hkv;
+  const int n_qt = (Lc + kT - 1) / kT;
+  const int U = G * n_qt;
+  const Attn2Tile t0 = attn2_tile(2 * blockIdx.x, U, G, n_qt, b * Hq + g * G, Lc, n_cache);
+  const Attn2Tile t1 = attn2_tile(2 * blockIdx.x + 1, U, G, n_qt, b * Hq + g * G, Lc, n_cache);
+  const int kv_head = b * Hkv + g;
+  const int n_kt0 = t0.n_kt, n_kt1 = t1.n_kt;  // n_kt0 >= n_kt1
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(q_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(k_full + s, 1);
+      ptx::mbar_init(k_empty + s, 1);
+      ptx::mbar_init(v_full + s, 1);
+      ptx::mbar_init(v_empty + s, 1);
+      ptx::mbar_init(s_full + s, 1);
+      ptx::mbar_init(p_ready + s, 128);
+      ptx::mbar_init(o_full + s, 1);
+    }
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp == 9) {
+    ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp >= 8) {
+    ptx::setmaxnreg_dec<56>();
+    if (warp == 8 && lane == 0) {
+      ptx::prefetch_tmap(&tmQ);
+      ptx::prefetch_tmap(&tmK);
+      ptx::prefetch_tmap(&tmV);
+      ptx::mbar_expect_tx(q_full, n_kt1 ? 2 * kTileBytes : kTileBytes);
+      ptx::tma_load_3d(sQ, &tmQ, q_full, 0, t0.row0, t0.head);
+      ptx::tma_load_3d(sQ + kHalfBytes, &tmQ, q_full, 64, t0.row0, t0.head);
+      if (n_kt1) {
+        ptx::tma_load_3d(sQ + kTileBytes, &tmQ, q_full, 0, t1.row0, t1.head);
+        ptx::tma_load_3d(sQ + kTileBytes + kHalfBytes, &tmQ, q_full, 64, t1.row0, t1.head);
+      }
+      int issued_k = 0, issued_v = 0;
+      for (int j = 0; j < n_kt0; ++j) {
+        const int s = j & 1, ph = (j >> 1) & 1;
+        if (!ptx::mbar_wait(k_empty + s, ph ^ 1, abort_flag)) break;
+        ptx::mbar_expect_tx(k_full + s, kTileBytes);
+        ptx::tma_load_3d(sK + s * kTileBytes, &tmK, k_full + s, 0, j * kT, kv_head);
+        ptx::tma_load_3d(sK + s * kTileBytes + kHalfBytes, &tmK, k_full + s, 64, j * kT, kv_head);
+        issued_k = j + 1;
+        if (!ptx::mbar_wait(v_empty + s, ph ^ 1, abort_flag)) break;
+        ptx::mbar_expect_tx(v_full + s, kTileBytes);
+        ptx::tma_load_3d(sV + s * kTileBytes, &tmV, v_full + s, 0, j * kT, kv_head);
+        ptx::tma_load_3d(sV + s * kTileBytes + kHalfBytes, &tmV, v_full + s, 64, j * kT, kv_head);
+        issued_v = j + 1;
+      }
+      if (*abort_flag) {  // let copies in flight land before the block's shared memory is released
+        volatile int ignore = 0;
+        ptx::mbar_wait(q_full, 0, &ignore);
+        for (int u = 1; u <= 2; ++u) {
+          if (issued_k >= u) ptx::mbar_wait(k_full + ((issued_k - u) & 1), ((issued_k - u) >> 1) & 1, &ignore);
+          if (issued_v >= u) ptx::mbar_wait(v_full + ((issued_v - u) & 1), ((issued_v - u) >> 1) & 1, &ignore);
+        }
+      }
+    } else if (warp == 9 && lane == 0) {
+      constexpr uint32_t idesc_pv = ptx::idesc_bf16(kT, kT, false, true);  // V is MN-major
+      const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK), aV = ptx::smem_u32(sV);
+      const uint32_t tS0 = tmem_base, tO0 = tmem_base + 128, tS1 = tmem_base + 256, tO1 = tmem_base + 384;
+      bool ok = ptx::mbar_wait(q_full, 0, abort_flag) && ptx::mbar_wait(k_full, 0, abort_flag);
+      if (ok) {
+        ptx::tc_fence_after();
+        issue_kmajor_128x128x128(tS0, aQ, aK);
+        ptx::mma_commit(s_full + 0);
+        if (n_kt1) {
+          issue_kmajor_128x128x128(tS1, aQ + kTileBytes, aK);
+          ptx::mma_commit(s_full + 1);
+        }
+        ptx::mma_commit(k_empty + 0);
+      }
+      for (int j = 0; ok && j < n_kt0; ++j) {
+        const int s = j & 1, ph = (j >> 1) & 1;
+        const int s1 = (j + 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+        // tile 0: O0 += P0 V[j], then S0 = Q0 K[j+1]^T
+        if (!ptx::mbar_wait(p_ready + 0, j & 1, abort_flag)) break;
+        if (!ptx::mbar_wait(v_full + s, ph, abort_flag)) break;
+        ptx::tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          ptx::mma_ts(tO0, tS0 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
+                      idesc_pv, (j > 0) || (k > 0));
+        if (j + 1 < n_kt0) {
+          if (!ptx::mbar_wait(k_full + s1, ph1, abort_flag)) break;
+          ptx::tc_fence_after();
+          issue_kmajor_128x128x128(tS0, aQ, aK + s1 * kTileBytes);
+          ptx::mma_commit(s_full + 0);
+        } else {
+          ptx::mma_commit(o_full + 0);
+        }
+        // tile 1
+        if (j < n_kt1) {
+          if (!ptx::mbar_wait(p_ready + 1, j & 1, abort_flag)) break;
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            ptx::mma_ts(tO1, tS1 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
+                        idesc_pv, (j > 0) || (k > 0));
+        }
+        ptx::mma_commit(v_empty + s);
+        if (j + 1 < n_kt1) {
+          issue_kmajor_128x128x128(tS1, aQ + kTileBytes, aK + s1 * kTileBytes);
+          ptx::mma_commit(s_full + 1);
+        } else if (j + 1 == n_kt1) {
+          ptx::mma_commit(o_full + 1);
+        }
+        if (j + 1 < n_kt0) ptx::mma_commit(k_empty + s1);
+      }
+    }
+  } else {
+    ptx::setmaxnreg_inc<224>();
+    const int t = warp >> 2;                      // which tile this warpgroup serves
+    const Attn2Tile tile = t ? t1 : t0;
+    const int sub = warp & 3;                     // TMEM sub-partition of this warp
+    const int r = 32 * sub + lane;                // row of the tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)(32 * sub) << 16;
+    const uint32_t tS = tmem_base + 256 * t + lane_addr, tO = tS + 128;
+    const int row = tile.row0 + r;
+    const int lim = n_cache + row;                // last visible key of this row
+    float m = -INFINITY, l0 = 0.f, l1 = 0.f;
+    bool ok = tile.n_kt > 0;
+    for (int j = 0; j < tile.n_kt; ++j) {
+      if (!ptx::mbar_wait(s_full + t, j & 1, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      uint32_t v[128];
+      ptx::tmem_ld128(tS, v);
+      const int key0 = j * kT;
+      if (key0 + kT - 1 > n_cache + tile.row0) {  // the walk reaches this tile's diagonal
+        const int thr = lim - key0;               // columns past thr are invisible to this row
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i > thr) v[i] = 0xff800000u;        // -inf
+      }
+      float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]);
+#pragma unroll
+      for (int i = 2; i < 128; i += 4) {
+        mx0 = ptx::max3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+        if (i + 3 < 128) mx1 = ptx::max3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+      }
+      const float m_new = fmaxf(m, fmaxf(mx0, mx1) * scale_log2);
+      if (j == 0) {
+        m = m_new;  // key 0 is visible to every row, so m is finite from here on
+      } else {
+        const bool grow = m_new > m + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
+          if (grow) m = m_new;
+          l0 *= alpha;
+          l1 *= alpha;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            ptx::tmem_ld32(tO + 32 * c, o);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            ptx::tmem_st32(tO + 32 * c, o);
+          }
+          ptx::tmem_st_wait();
+        }
+      }
+      const float neg_m = -m;
+      uint32_t pk[64];
+#pragma unroll
+      for (int i = 0; i < 128; i += 2) {
+        float x0, x1;
+        ptx::fma2(x0, x1, __uint_as_float(v[i]), __uint_as_float(v[i + 1]), scale_log2, neg_m);
+        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);  // ex2(-inf) = 0 for masked columns
+        ptx::add2(l0, l1, p0, p1);
+        pk[i >> 1] = ptx::pack_bf16(p0, p1);
+      }
+      ptx::tmem_st64(tS, pk);
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(p_ready + t);
+    }
+    if (ok && ptx::mbar_wait(o_full + t, 0, abort_flag)) {
+      ptx::tc_fence_after();
+      const float l = l0 + l1;
+      const float inv = 1.0f / l;
+      __nv_bfloat16* op = out + ((long long)tile.head * Lc + row) * kT;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        ptx::tmem_ld32(tO + 32 * c, o);
+        if (row < Lc) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 w;
+            w.x = ptx::pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+            w.y = ptx::pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            w.z = ptx::pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+            w.w = ptx::pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(op + 32 * c + i) = w;
+          }
+        }
+      }
+      if (row < Lc) lse[(long long)tile.head * Lc + row] = (m + log2f(l)) * kLn2;
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+}
+
 // Enumerates the (query head of the group, 128-row query tile of the window)
 // pairs a key tile has to visit, skipping tiles none of whose rows sees it.
 struct ScoreTiles {
@@ -429,10 +706,20 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
     q.flags |= REFORM_NO_SCORE;
     rc = launch_chunk_simt(&q, lse, scale, st);
     if (rc != REFORM_OK) return rc;
-  } else {
+  } else if (mode == 3) {
     cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
     dim3 grid((p->Lc + kT - 1) / kT, p->B * p->Hq);
     attn_sm100_kernel<<<grid, kSm100Threads, kAttnSmemBytes, st>>>(
+        tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
+        p->dev_status);
+    count_launch();
+    rc = check_launch();
+    if (rc != REFORM_OK) return rc;
+  } else {
+    cudaFuncSetAttribute(attn2_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttn2SmemBytes);
+    const int units = (p->Hq / p->Hkv) * ((p->Lc + kT - 1) / kT);
+    dim3 grid((units + 1) / 2, p->B * p->Hkv);
+    attn2_sm100_kernel<<<grid, kAttn2Threads, kAttn2SmemBytes, st>>>(
         tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
         p->dev_status);
     count_launch();
