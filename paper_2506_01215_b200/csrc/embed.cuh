@@ -91,11 +91,90 @@ embed_append_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, in
   }
 }
 
+
+// Fast path for vectors of 4, 8, 16 or 32 sixteen-byte chunks (bf16 d = 32..256,
+// fp32 d = 16..128): LP lanes own one vector, a warp works on 32/LP vectors at
+// a time and keeps four such groups in flight.
+template <typename T, int LP>
+__global__ void __launch_bounds__(256)
+embed_append_vec_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, int E,
+                        long long N_cap, long long token_offset, float eps) {
+  constexpr int VPW = 32 / LP, U = 4, EPC = 16 / (int)sizeof(T);
+  const int lane = threadIdx.x & 31;
+  const int sub = lane % LP, which = lane / LP;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long items = (long long)B * Lc * sel.n_sel;
+  for (long long it0 = warp * (VPW * U); it0 < items; it0 += n_warps * (VPW * U)) {
+    uint4 x[U];
+    T* y[U];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      long long it = it0 + u * VPW + which;
+      ok[u] = it < items;
+      x[u] = make_uint4(0, 0, 0, 0);
+      y[u] = nullptr;
+      if (ok[u]) {
+        int s = (int)(it % sel.n_sel);
+        long long bt = it / sel.n_sel;
+        int t = (int)(bt % Lc);
+        int b = (int)(bt / Lc);
+        const T* src = reinterpret_cast<const T*>(sel.src[s]) +
+                       (((long long)b * sel.H[s] + sel.head[s]) * Lc + t) * d;
+        x[u] = __ldcs(reinterpret_cast<const uint4*>(src) + sub);
+        y[u] = bank + ((long long)b * N_cap + token_offset + t) * E + (long long)sel.slot[s] * d + sub * EPC;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      float f[EPC];
+      const T* e = reinterpret_cast<const T*>(&x[u]);
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < EPC; ++i) {
+        f[i] = to_float(e[i]);
+        ss = fmaf(f[i], f[i], ss);
+      }
+#pragma unroll
+      for (int o = LP / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float nrm = fmaxf(sqrtf(ss), eps);
+      uint4 w;
+      T* o4 = reinterpret_cast<T*>(&w);
+#pragma unroll
+      for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>(f[i] / nrm);
+      if (ok[u]) __stcs(reinterpret_cast<uint4*>(y[u]), w);
+    }
+  }
+}
+
 template <typename T>
 inline int launch_embed(const EmbedSel& sel, void* bank, int B, int Lc, int d, int E,
                         long long N_cap, long long token_offset, float eps, cudaStream_t st) {
   long long items = (long long)B * Lc * sel.n_sel;
   if (items == 0) return REFORM_OK;
+  const int chunks = d * (int)sizeof(T) / 16;
+  const bool vec_ok = (d * sizeof(T)) % 16 == 0 && (chunks == 4 || chunks == 8 || chunks == 16 || chunks == 32);
+  if (vec_ok) {
+    long long per_warp = (32 / chunks) * 4;
+    long long blocks = (items + 8 * per_warp - 1) / (8 * per_warp);
+    long long cap = (long long)kNumSMs * 8;
+    int grid = (int)(blocks < cap ? blocks : cap);
+#define REFORM_EMBED_CASE(LP)                                                                          \
+  case LP:                                                                                             \
+    embed_append_vec_kernel<T, LP><<<grid, 256, 0, st>>>(sel, (T*)bank, B, Lc, d, E, N_cap,           \
+                                                         token_offset, eps);                           \
+    break;
+    switch (chunks) {
+      REFORM_EMBED_CASE(4)
+      REFORM_EMBED_CASE(8)
+      REFORM_EMBED_CASE(16)
+      REFORM_EMBED_CASE(32)
+    }
+#undef REFORM_EMBED_CASE
+    count_launch();
+    return check_launch();
+  }
   long long blocks = (items + 7) / 8;  // 8 warps per block
   long long cap = (long long)kNumSMs * 16;
   int grid = (int)(blocks < cap ? blocks : cap);

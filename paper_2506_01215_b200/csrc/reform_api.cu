@@ -151,7 +151,7 @@ int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream) {
   a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
   a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
   a.blocks_per_seg = L.blocks_per_seg;
-  rc = launch_select(a, segs, nullptr, nullptr, 0, st);
+  rc = launch_select(a, segs, nullptr, nullptr, 0, ws, L, p->dev_status, st);
   if (rc != REFORM_OK) return rc;
   return launch_evict_compact(p->k_src, p->v_src, p->k_dst, p->v_dst, p->score_src, p->score_dst,
                               p->pos_src, p->pos_dst, kept, p->budget, segs, n_kept, p->cap_src,
@@ -265,7 +265,7 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
   a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
   a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
   a.blocks_per_seg = L.blocks_per_seg;
-  return launch_select(a, p->B, ts, pooled, (p->pool_window - 1) / 2, st);
+  return launch_select(a, p->B, ts, pooled, (p->pool_window - 1) / 2, ws, L, p->dev_status, st);
 }
 
 /* --------------------------------------------------------------- gather */

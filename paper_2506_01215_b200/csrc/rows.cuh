@@ -49,8 +49,8 @@ inline int launch_gather(const uint4* src, const int32_t* idx, uint4* dst, int B
   long long total = (long long)B * k;
   if (total == 0) return REFORM_OK;
   int vec = (int)(row_bytes / 16);
-  int lanes = 1;
-  while (lanes < vec && lanes < kRowThreads) lanes <<= 1;  // power of two, <= 256
+  int lanes = 1;  // power of two, <= 256, about four 16-byte chunks per lane so four loads are in flight
+  while (4 * lanes < vec && lanes < kRowThreads) lanes <<= 1;
   long long rows_per_block = kRowThreads / lanes;
   long long blocks = (total + rows_per_block - 1) / rows_per_block;
   long long cap = (long long)kNumSMs * 16;
@@ -100,7 +100,16 @@ evict_compact_kernel(const uint4* __restrict__ k_src, const uint4* __restrict__ 
     int j = kept[(long long)s * kept_stride + rank];
     const uint4* sp = src + ((long long)s * cap_src + j) * vec;
     uint4* dp = dst + ((long long)s * cap_dst + rank) * vec;
-    for (int c = lane; c < vec; c += LANES) __stcs(dp + c, __ldcs(sp + c));
+    int c = lane;
+    for (; c + 3 * LANES < vec; c += 4 * LANES) {
+      uint4 a0 = __ldcs(sp + c), a1 = __ldcs(sp + c + LANES), a2 = __ldcs(sp + c + 2 * LANES),
+            a3 = __ldcs(sp + c + 3 * LANES);
+      __stcs(dp + c, a0);
+      __stcs(dp + c + LANES, a1);
+      __stcs(dp + c + 2 * LANES, a2);
+      __stcs(dp + c + 3 * LANES, a3);
+    }
+    for (; c < vec; c += LANES) __stcs(dp + c, __ldcs(sp + c));
     if (blockIdx.y == 0 && lane == 0) {
       if (score_dst) score_dst[(long long)s * cap_dst + rank] = score_src[(long long)s * cap_src + j];
       if (pos_dst) pos_dst[(long long)s * cap_dst + rank] = pos_src[(long long)s * cap_src + j];
@@ -117,7 +126,7 @@ inline int launch_evict_compact(const void* k_src, const void* v_src, void* k_ds
   if (total == 0) return REFORM_OK;
   int vec = row_bytes / 16;
   int lanes = 1;
-  while (lanes < vec && lanes < 32) lanes <<= 1;
+  while (4 * lanes < vec && lanes < 32) lanes <<= 1;
   long long rows_per_block = kRowThreads / lanes;
   long long blocks = (total + rows_per_block - 1) / rows_per_block;
   long long cap = (long long)kNumSMs * 8;

@@ -32,7 +32,7 @@ struct SelState {      // per segment, in the workspace
 };
 
 struct SelLayout {  // offsets into the workspace, per call
-  size_t state, hist, blockcnt, total;
+  size_t state, hist, ctl, zero_bytes, blockcnt, total;  // [state, hist, ctl] are contiguous
   int blocks_per_seg;
 };
 
@@ -45,6 +45,9 @@ inline SelLayout sel_layout(int segs, long long n_max) {
   off += align_up(sizeof(SelState) * segs, 256);
   L.hist = off;
   off += align_up(sizeof(uint32_t) * 3 * kSelBins * segs, 256);
+  L.ctl = off;
+  off += align_up(16 * (size_t)segs, 256);
+  L.zero_bytes = off;  // everything up to here is cleared at the start of a fused launch
   L.blockcnt = off;
   off += align_up(sizeof(uint2) * 2 * (size_t)L.blocks_per_seg * segs, 256);
   L.total = off;
@@ -309,12 +312,235 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(SelArgs a) {
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// Single-launch form of the same selection for inputs whose blocks are all
+// resident at once (cooperative launch): the three histogram passes, the count
+// and the ordered write run in one kernel, separated by per-segment barriers
+// over a global counter, and every thread keeps its four keys in registers
+// from the first pass to the last.  Each block re-derives the digit decisions
+// from the global histograms itself, so no block depends on another block's
+// private state.  The barrier wait is bounded: a block that gives up sets
+// REFORM_DEV_TIMEOUT in *dev_status and the launch winds down.
+// ---------------------------------------------------------------------------
+struct SelFusedCtl {   // per segment, zeroed before the launch
+  uint32_t arrived;    // barrier counter (monotonic)
+  uint32_t abort;
+  uint32_t pad[2];
+};
+
+__device__ __forceinline__ bool sel_seg_barrier(SelFusedCtl* ctl, uint32_t expected, int32_t* dev_status) {
+  __shared__ int failed;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    failed = 0;
+    __threadfence();
+    atomicAdd(&ctl->arrived, 1u);
+    const long long t0 = clock64();
+    while (atomicAdd(&ctl->arrived, 0u) < expected) {
+      if (*reinterpret_cast<volatile uint32_t*>(&ctl->abort) || clock64() - t0 > 400000000LL) {
+        atomicExch(&ctl->abort, 1u);
+        if (dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+        failed = 1;
+        break;
+      }
+    }
+    __threadfence();
+  }
+  __syncthreads();
+  return failed == 0;
+}
+
+// Walk the 2048 bins of one pass from the top; every thread returns the same (bin, remaining).
+__device__ __forceinline__ void sel_find_bin_local(const uint32_t* hist, uint32_t remaining, uint32_t* scratch,
+                                                   uint32_t* result, uint32_t& bin_out, uint32_t& rem_out) {
+  int b0 = kSelBins - 1 - 2 * (int)threadIdx.x;
+  uint32_t c0 = __ldcg(hist + b0), c1 = __ldcg(hist + b0 - 1);
+  uint32_t total;
+  uint32_t before = block_excl_scan(c0 + c1, scratch, total);
+  if (threadIdx.x == 0) { result[0] = kSelBins - 1; result[1] = 0; }  // remaining == 0: above every key
+  __syncthreads();
+  if (before < remaining && remaining <= before + c0 + c1) {
+    if (remaining <= before + c0) { result[0] = b0; result[1] = remaining - before; }
+    else { result[0] = b0 - 1; result[1] = remaining - before - c0; }
+  }
+  __syncthreads();
+  bin_out = result[0];
+  rem_out = result[1];
+  __syncthreads();
+}
+
+template <bool POOL>
+__global__ void __launch_bounds__(kSelThreads)
+sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
+                 float* __restrict__ pooled_out, int radius, int32_t* dev_status) {
+  extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
+  __shared__ uint32_t hist[kSelBins];
+  __shared__ uint32_t scratch[33];
+  __shared__ uint32_t result[2];
+  const int seg = blockIdx.y, tid = threadIdx.x;
+  const uint32_t nblk = gridDim.x;
+  SelFusedCtl* ctl = ctl_all + seg;
+  const long long base = (long long)blockIdx.x * kSelTile;
+  uint32_t key[kSelPerThread];
+  bool cand[kSelPerThread];
+
+  if (POOL) {
+    const int span = kSelTile + 2 * radius;
+    float* cur = tile;
+    float* nxt = tile + span;
+    const float* src = ts + (long long)seg * a.stride;
+    for (int i = tid; i < span; i += kSelThreads) {
+      long long g = base - radius + i;
+      cur[i] = (g >= 0 && g < a.n) ? src[g] : -INFINITY;
+    }
+    __syncthreads();
+    const int window = 2 * radius + 1;
+    int len = 1;
+    while (2 * len <= window) {
+      for (int i = tid; i < span; i += kSelThreads) {
+        float v = cur[i];
+        if (i + len < span) v = fmaxf(v, cur[i + len]);
+        nxt[i] = v;
+      }
+      __syncthreads();
+      float* t = cur; cur = nxt; nxt = t;
+      len *= 2;
+    }
+    float* dst = pooled_out + (long long)seg * a.stride;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+      int i = j * kSelThreads + tid;
+      long long g = base + i;
+      cand[j] = g >= a.lo && g < a.hi;
+      key[j] = 0;
+      if (g < a.n) {
+        float v = fmaxf(cur[i], cur[i + window - len]);
+        dst[g] = v;
+        key[j] = float_to_key(v);
+      }
+    }
+  } else {
+    const float* src = a.vals + (long long)seg * a.stride;
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j) {
+      long long g = base + j * kSelThreads + tid;
+      cand[j] = g >= a.lo && g < a.hi;
+      key[j] = cand[j] ? float_to_key(src[g]) : 0u;
+    }
+  }
+
+  uint32_t prefix = 0, remaining = (uint32_t)a.m;
+  uint32_t phase = 0;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    int shift;
+    uint32_t dmask, pmask;
+    sel_pass_params(pass, shift, dmask, pmask);
+    for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kSelPerThread; ++j)
+      if (cand[j] && (key[j] & pmask) == prefix) atomicAdd(&hist[(key[j] >> shift) & dmask], 1u);
+    __syncthreads();
+    uint32_t* gh = a.hist + ((size_t)seg * 3 + pass) * kSelBins;
+    for (int i = tid; i < kSelBins; i += kSelThreads) {
+      uint32_t c = hist[i];
+      if (c) atomicAdd(gh + i, c);
+    }
+    if (!sel_seg_barrier(ctl, ++phase * nblk, dev_status)) return;
+    uint32_t bin, rem;
+    sel_find_bin_local(gh, remaining, scratch, result, bin, rem);
+    prefix |= bin << shift;
+    remaining = rem;
+  }
+  const uint32_t thr = prefix, need_eq = remaining;
+
+  // per-block counts in index order, then offsets from the blocks before this one
+  uint32_t is_gt[kSelPerThread], is_eq[kSelPerThread];
+  uint32_t gt = 0, eq = 0;
+#pragma unroll
+  for (int j = 0; j < kSelPerThread; ++j) {
+    is_gt[j] = cand[j] && key[j] > thr;
+    is_eq[j] = cand[j] && key[j] == thr;
+    gt += is_gt[j];
+    eq += is_eq[j];
+  }
+  uint32_t tot_gt, tot_eq;
+  block_excl_scan(gt, scratch, tot_gt);
+  block_excl_scan(eq, scratch, tot_eq);
+  uint2* cnt = a.blockcnt + (size_t)seg * 2 * a.blocks_per_seg;
+  if (tid == 0) cnt[blockIdx.x] = make_uint2(tot_gt, tot_eq);
+  if (!sel_seg_barrier(ctl, ++phase * nblk, dev_status)) return;
+  uint32_t pg = 0, pe = 0;
+  for (int bb = tid; bb < (int)blockIdx.x; bb += kSelThreads) {
+    uint2 c = __ldcg(cnt + bb);
+    pg += c.x;
+    pe += c.y;
+  }
+  uint32_t run_gt, run_eq, dummy;
+  block_excl_scan(pg, scratch, run_gt);
+  block_excl_scan(pe, scratch, run_eq);
+  (void)dummy;
+
+  int32_t* out = a.out + (long long)seg * a.out_stride;
+#pragma unroll
+  for (int j = 0; j < kSelPerThread; ++j) {
+    uint32_t tg, te;
+    uint32_t sg = block_excl_scan(is_gt[j], scratch, tg);
+    uint32_t se = block_excl_scan(is_eq[j], scratch, te);
+    uint32_t gt_before = run_gt + sg, eq_before = run_eq + se;
+    if (is_gt[j] || (is_eq[j] && eq_before < need_eq)) {
+      uint32_t pos = a.lo + gt_before + (eq_before < need_eq ? eq_before : need_eq);
+      out[pos] = (int32_t)(base + j * kSelThreads + tid);
+    }
+    run_gt += tg;
+    run_eq += te;
+  }
+  if (blockIdx.x == 0) {
+    for (int i = tid; i < a.lo; i += kSelThreads) out[i] = i;
+    int tail = a.n - a.hi;
+    for (int i = tid; i < tail; i += kSelThreads) out[a.lo + a.m + i] = a.hi + i;
+  }
+}
+
 // Enqueue the whole selection.  If ts != nullptr the first pass pools ts with
 // the given radius into pooled (which must then be a.vals).
+// Blocks of sel_fused_kernel that can be resident at once on this device (0 if unknown).
+template <bool POOL>
+inline int sel_fused_capacity(size_t smem) {
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sel_fused_kernel<POOL>, kSelThreads, smem) !=
+      cudaSuccess)
+    return 0;
+  return sms * per_sm;
+}
+
 inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, int radius,
-                         cudaStream_t st) {
+                         void* ws_base, const SelLayout& L, int32_t* dev_status, cudaStream_t st) {
   if (segs == 0) return REFORM_OK;
   dim3 grid(a.blocks_per_seg, segs);
+  {
+    const size_t smem = ts ? sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius) : 0;
+    if (ts) cudaFuncSetAttribute(sel_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int capacity = ts ? sel_fused_capacity<true>(smem) : sel_fused_capacity<false>(smem);
+    if ((long long)a.blocks_per_seg * segs <= capacity) {
+      if (cudaMemsetAsync(ws_base, 0, L.zero_bytes, st) != cudaSuccess) return check_launch();
+      SelFusedCtl* ctl = reinterpret_cast<SelFusedCtl*>(reinterpret_cast<char*>(ws_base) + L.ctl);
+      void* args[] = {&a, &ctl, &ts, &pooled, &radius, &dev_status};
+      cudaError_t e = cudaLaunchCooperativeKernel(
+          ts ? (const void*)sel_fused_kernel<true> : (const void*)sel_fused_kernel<false>, grid,
+          dim3(kSelThreads), args, smem, st);
+      if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return REFORM_ERR_CUDA;
+      }
+      count_launch();
+      return check_launch();
+    }
+  }
   sel_init_kernel<<<segs, 256, 0, st>>>(a, segs);
   count_launch();
   if (ts) {

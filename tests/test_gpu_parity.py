@@ -144,6 +144,23 @@ def test_evict_matches_oracle_bit_exactly(B, Hkv, d, n_keys, budget, sink, recen
     assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept])
 
 
+def test_evict_many_segments_multi_launch_path():
+    """More blocks than can be resident at once: the selection falls back to
+    one launch per pass; results must not change."""
+    g = torch.Generator().manual_seed(4)
+    B, Hkv, n, d, budget = 48, 8, 4200, 4, 1000
+    k = torch.randn(B, Hkv, n, d, generator=g)
+    sc = (torch.rand(B, Hkv, n, generator=g) * 50).floor()   # many ties
+    ref = oracle.evict_topk(k, k, sc, n, budget, 16, 16, cap_dst=budget)
+    kd = torch.zeros(B, Hkv, budget, d, device=DEV)
+    vd = torch.zeros_like(kd)
+    sd = torch.zeros(B, Hkv, budget, device=DEV)
+    kept = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV)
+    R.evict_topk(k.to(DEV), k.to(DEV).clone(), sc.to(DEV), kd, vd, sd, n, budget, 16, 16, kept_idx=kept)
+    assert torch.equal(kept.cpu(), ref["kept_idx"])
+    assert torch.equal(kd.cpu(), ref["k"])
+
+
 def test_evict_without_optional_outputs():
     g = torch.Generator().manual_seed(1)
     k = torch.randn(1, 2, 600, 64, generator=g)
