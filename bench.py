@@ -72,6 +72,16 @@ def attn_flops(w, step):
     return 4 * w.B * w.Hq * w.d * attn_pairs(w, step)
 
 
+# DRAM bytes the attention kernel moved per algorithmic byte (Q + K + V + O) in the ncu capture of
+# the small case (profiles/attn2_sm100_kernel_lc8192.md): 174.7 MB / 201.3 MB.
+ATTN_DRAM_RATIO = 0.87
+
+
+def attn_bytes(w):
+    sz = 2 if w.dtype == torch.bfloat16 else 4
+    return w.B * sz * w.d * (2 * w.Hq * w.Lc + 2 * w.Hkv * (w.budget + w.Lc))
+
+
 def retrieval_gather_bytes(w):
     sz = 2 if w.dtype == torch.bfloat16 else 4
     return w.B * (w.N * w.E * sz + 2 * w.k * w.D * sz)
@@ -409,7 +419,10 @@ def main():
         "roofline": {"bound": "tensor", "kernel": "reform_chunk_step (attention + score pass)",
                      "achieved": achieved, "peak": pk["tflops"], "unit": "TFLOP/s",
                      "frac": achieved / pk["tflops"], "frac_of_nominal_2250": achieved / 2250.0,
-                     "traffic": None, "peak_source": pk["source"],
+                     "traffic": ATTN_DRAM_RATIO * attn_bytes(w), "traffic_unit": "bytes per launch (steps >= 1)",
+                     "traffic_source": ("ncu dram__bytes_read+write of the small-case capture in profiles/, "
+                                        "scaled by algorithmic bytes Q+K+V+O"),
+                     "peak_source": pk["source"],
                      "flops_counted": "4*Hq*d*visible pairs (QK^T and PV of unmasked pairs only)"},
         "gpu_launches": launches,
         "clocks": clocks,

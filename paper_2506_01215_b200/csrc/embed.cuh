@@ -102,24 +102,23 @@ embed_append_vec_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d
   constexpr int VPW = 32 / LP, U = 4, EPC = 16 / (int)sizeof(T);
   const int lane = threadIdx.x & 31;
   const int sub = lane % LP, which = lane / LP;
-  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long items = (long long)B * Lc * sel.n_sel;
-  for (long long it0 = warp * (VPW * U); it0 < items; it0 += n_warps * (VPW * U)) {
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t n_warps = (gridDim.x * blockDim.x) >> 5;
+  const uint32_t n_sel = (uint32_t)sel.n_sel;
+  const uint32_t items = (uint32_t)B * (uint32_t)Lc * n_sel;  // < 2^31, checked by the launcher
+  for (uint32_t it0 = warp * (VPW * U); it0 < items; it0 += n_warps * (VPW * U)) {
     uint4 x[U];
     T* y[U];
     bool ok[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      long long it = it0 + u * VPW + which;
+      const uint32_t it = it0 + u * VPW + which;
       ok[u] = it < items;
       x[u] = make_uint4(0, 0, 0, 0);
       y[u] = nullptr;
       if (ok[u]) {
-        int s = (int)(it % sel.n_sel);
-        long long bt = it / sel.n_sel;
-        int t = (int)(bt % Lc);
-        int b = (int)(bt / Lc);
+        const uint32_t bt = it / n_sel, s = it - bt * n_sel;
+        const uint32_t b = bt / (uint32_t)Lc, t = bt - b * (uint32_t)Lc;
         const T* src = reinterpret_cast<const T*>(sel.src[s]) +
                        (((long long)b * sel.H[s] + sel.head[s]) * Lc + t) * d;
         x[u] = __ldcs(reinterpret_cast<const uint4*>(src) + sub);
@@ -138,11 +137,11 @@ embed_append_vec_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d
       }
 #pragma unroll
       for (int o = LP / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float nrm = fmaxf(sqrtf(ss), eps);
+      const float inv = 1.0f / fmaxf(sqrtf(ss), eps);
       uint4 w;
       T* o4 = reinterpret_cast<T*>(&w);
 #pragma unroll
-      for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>(f[i] / nrm);
+      for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>(f[i] * inv);
       if (ok[u]) __stcs(reinterpret_cast<uint4*>(y[u]), w);
     }
   }
@@ -154,7 +153,8 @@ inline int launch_embed(const EmbedSel& sel, void* bank, int B, int Lc, int d, i
   long long items = (long long)B * Lc * sel.n_sel;
   if (items == 0) return REFORM_OK;
   const int chunks = d * (int)sizeof(T) / 16;
-  const bool vec_ok = (d * sizeof(T)) % 16 == 0 && (chunks == 4 || chunks == 8 || chunks == 16 || chunks == 32);
+  const bool vec_ok = (d * sizeof(T)) % 16 == 0 && items < (1LL << 31) &&
+                      (chunks == 4 || chunks == 8 || chunks == 16 || chunks == 32);
   if (vec_ok) {
     long long per_warp = (32 / chunks) * 4;
     long long blocks = (items + 8 * per_warp - 1) / (8 * per_warp);
