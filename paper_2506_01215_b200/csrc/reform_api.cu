@@ -14,6 +14,7 @@
 #endif
 #ifndef REFORM_NO_SM100
 #include "chunk_sm100.cuh"
+#include "retrieve_sm100.cuh"
 #endif
 
 namespace reform {
@@ -245,7 +246,14 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
   if (!ts) { ts = reinterpret_cast<float*>(ws + off); off += retrieve_score_bytes(p); }
   float* pooled = p->pooled_score_out;
   if (!pooled) { pooled = reinterpret_cast<float*>(ws + off); off += retrieve_score_bytes(p); }
-  rc = launch_scan(p->dtype, p->bank, p->queries, ts, p->B, p->N, p->N_cap, p->E, p->nq, p->scale, st);
+  rc = REFORM_ERR_UNSUPPORTED;
+#ifndef REFORM_NO_SM100
+  if (p->dtype == REFORM_BF16 && !getenv("REFORM_SCAN_NO_TCGEN05"))
+    rc = launch_scan_sm100(p->bank, p->queries, ts, p->B, p->N, p->N_cap, p->E, p->nq, p->scale,
+                           p->dev_status, st);
+#endif
+  if (rc == REFORM_ERR_UNSUPPORTED)
+    rc = launch_scan(p->dtype, p->bank, p->queries, ts, p->B, p->N, p->N_cap, p->E, p->nq, p->scale, st);
   if (rc != REFORM_OK) return rc;
   SelArgs a;
   a.vals = pooled;
