@@ -52,7 +52,8 @@ enum {
   REFORM_ERR_INVALID_ARG = -1, /* NULL pointer, bad size, bad struct_size, misaligned pointer */
   REFORM_ERR_UNSUPPORTED = -2, /* dtype / head dimension the kernels do not cover */
   REFORM_ERR_WORKSPACE = -3,   /* workspace missing or too small */
-  REFORM_ERR_CUDA = -4         /* a CUDA call failed; see reform_last_cuda_error() */
+  REFORM_ERR_CUDA = -4,        /* a CUDA call failed; see reform_last_cuda_error() */
+  REFORM_ERR_TOO_LARGE = -5    /* problem exceeds the built-in scratch of a *_static entry point */
 };
 
 enum { REFORM_F32 = 0, REFORM_BF16 = 1 };
@@ -160,6 +161,39 @@ typedef struct reform_evict_params {
 
 size_t reform_evict_topk_workspace_size(const reform_evict_params* p);
 int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_evict_topk_static -- the paper has no counterpart; this is a
+ * packaging variant of reform_evict_topk for callers that cannot allocate
+ * device memory and so have no workspace to pass: for example a serving
+ * process that handed all of HBM to its KV-cache pool at start-up (a later
+ * cudaMalloc would simply fail), or a latency-critical loop in which the
+ * device-wide synchronisation that cudaMalloc / cudaFree imply is not allowed.
+ *
+ * Same arguments, same results and same kernels as reform_evict_topk, except
+ * that p->workspace and p->workspace_bytes are ignored: the scratch (the
+ * selection histograms and counters, and the kept-index list when p->kept_idx
+ * is NULL) lives in a fixed array inside the library, REFORM_EVICT_STATIC_BYTES
+ * large, that every GPU which loads the library holds until the process exits.
+ * The call allocates nothing and frees nothing.
+ *
+ * Limits: B * Hkv <= REFORM_EVICT_STATIC_MAX_SEGS, n_keys <=
+ * REFORM_EVICT_STATIC_MAX_KEYS, budget <= REFORM_EVICT_STATIC_MAX_BUDGET;
+ * anything larger returns REFORM_ERR_TOO_LARGE and launches nothing.
+ *
+ * The first call on each device looks up the array's device address (with
+ * that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents (the call clears what must start at zero): two calls that overlap
+ * on the GPU -- different streams, or different host threads -- race on it.
+ * Calls on one stream are safe.
+ * ------------------------------------------------------------------------ */
+#define REFORM_EVICT_STATIC_MAX_SEGS 32
+#define REFORM_EVICT_STATIC_MAX_KEYS 65536
+#define REFORM_EVICT_STATIC_MAX_BUDGET 16384
+#define REFORM_EVICT_STATIC_BYTES (3u << 20)
+
+int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------
  * reform_embed_append -- Sec. 3.2 "Combining multiple heads":

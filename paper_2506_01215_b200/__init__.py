@@ -21,7 +21,8 @@ LIB_PATH = os.path.join(_HERE, "libreform.so")
 F32, BF16 = 0, 1
 SCORE_ACCUMULATE, NO_SCORE, FORCE_SIMT = 1, 2, 4
 STATE_Q, STATE_K, STATE_V = 0, 1, 2
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
+EVICT_STATIC_MAX_SEGS, EVICT_STATIC_MAX_KEYS, EVICT_STATIC_MAX_BUDGET = 32, 65536, 16384
 DEV_TIMEOUT, DEV_BAD_INDEX = 1, 2
 MAX_SEL = 16
 
@@ -74,7 +75,7 @@ class GatherParams(ctypes.Structure):
 
 EXPORTS = (
     "reform_chunk_step", "reform_chunk_step_workspace_size", "reform_evict_topk",
-    "reform_evict_topk_workspace_size", "reform_embed_append", "reform_retrieve_topk",
+    "reform_evict_topk_workspace_size", "reform_evict_topk_static", "reform_embed_append", "reform_retrieve_topk",
     "reform_retrieve_topk_workspace_size", "reform_gather", "reform_status_string",
     "reform_last_cuda_error", "reform_version", "reform_kernel_launch_count",
 )
@@ -106,6 +107,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ctypes.c_int
             getattr(L, name + "_workspace_size").argtypes = [ctypes.POINTER(ptype)]
             getattr(L, name + "_workspace_size").restype = _sz
+        L.reform_evict_topk_static.argtypes = [ctypes.POINTER(EvictParams), _vp]
+        L.reform_evict_topk_static.restype = ctypes.c_int
         L.reform_embed_append.argtypes = [ctypes.POINTER(EmbedParams), _vp]
         L.reform_embed_append.restype = ctypes.c_int
         L.reform_gather.argtypes = [ctypes.POINTER(GatherParams), _vp]
@@ -202,6 +205,25 @@ def evict_topk(k_src, v_src, score_src, k_dst, v_dst, score_dst, n_keys: int, bu
     return n_kept.value
 
 
+def evict_topk_static(k_src, v_src, score_src, k_dst, v_dst, score_dst, n_keys: int, budget: int,
+                      n_sink: int, n_recent: int, *, pos_src=None, pos_dst=None, kept_idx=None,
+                      stream=None) -> int:
+    """reform_evict_topk_static: reform_evict_topk for callers that cannot allocate device memory
+    (no workspace argument; the library's built-in scratch is used, and neither this wrapper nor the
+    call allocates anything).  Raises ReformError(ERR_TOO_LARGE) beyond B*Hkv <= 32, n_keys <= 65536,
+    budget <= 16384.  Calls that overlap on the GPU share the scratch and race; keep them on one
+    stream.  Returns n_kept."""
+    B, Hkv, cap_src, d = k_src.shape
+    cap_dst = k_dst.shape[2]
+    n_kept = ctypes.c_int32(0)
+    p = EvictParams(ctypes.sizeof(EvictParams), _dtype_code(k_src), B, Hkv, d, int(n_keys), cap_src,
+                    cap_dst, int(budget), int(n_sink), int(n_recent), _ptr(k_src), _ptr(v_src),
+                    _ptr(score_src), _ptr(pos_src), _ptr(k_dst), _ptr(v_dst), _ptr(score_dst),
+                    _ptr(pos_dst), _ptr(kept_idx), ctypes.addressof(n_kept), None, 0, None)
+    _check("reform_evict_topk_static", lib().reform_evict_topk_static(ctypes.byref(p), _stream(stream)))
+    return n_kept.value
+
+
 def embed_append(bank, token_offset: int, sel: Sequence[Tuple[int, int, int]], *, q_state=None,
                  k_state=None, v_state=None, eps: float = 0.0, stream=None):
     """reform_embed_append: bank [B,N_cap,E]; sel = [(kind, head, slot), ...]."""
@@ -248,6 +270,7 @@ def gather(src, idx, dst, *, dev_status=None, stream=None):
 # the C entry points' own names, for callers that prefer them
 reform_chunk_step = chunk_step
 reform_evict_topk = evict_topk
+reform_evict_topk_static = evict_topk_static
 reform_embed_append = embed_append
 reform_retrieve_topk = retrieve_topk
 reform_gather = gather

@@ -159,6 +159,53 @@ int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream) {
                               p->cap_dst, (int)(p->d * elem_size(p->dtype)), st);
 }
 
+/* ------------------------------------------ evict without a workspace */
+
+// Scratch of reform_evict_topk_static.  In host code this name is only a
+// handle for cudaGetSymbolAddress; the kernels get the device address.
+static __device__ __align__(256) unsigned char g_evict_static_scratch[REFORM_EVICT_STATIC_BYTES];
+
+// Device address of the scratch array on the current device, looked up once per device.
+static int evict_static_scratch(void** out) {
+  constexpr int kMaxDevices = 64;
+  static std::atomic<void*> cache[kMaxDevices];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    g_last_cuda_error = (int)(e != cudaSuccess ? e : cudaErrorInvalidDevice);
+    return REFORM_ERR_CUDA;
+  }
+  void* ptr = cache[dev].load(std::memory_order_acquire);
+  if (!ptr) {
+    e = cudaGetSymbolAddress(&ptr, g_evict_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      g_last_cuda_error = (int)e;
+      return REFORM_ERR_CUDA;
+    }
+    cache[dev].store(ptr, std::memory_order_release);
+  }
+  *out = ptr;
+  return REFORM_OK;
+}
+
+int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t stream) {
+  int rc = validate_evict(p);
+  if (rc != REFORM_OK) return rc;
+  if ((long long)p->B * p->Hkv > REFORM_EVICT_STATIC_MAX_SEGS || p->n_keys > REFORM_EVICT_STATIC_MAX_KEYS ||
+      p->budget > REFORM_EVICT_STATIC_MAX_BUDGET)
+    return REFORM_ERR_TOO_LARGE;
+  reform_evict_params q = *p;
+  q.workspace = nullptr;
+  q.workspace_bytes = 0;
+  if (reform_evict_topk_workspace_size(&q) > REFORM_EVICT_STATIC_BYTES) return REFORM_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  rc = evict_static_scratch(&scratch);
+  if (rc != REFORM_OK) return rc;
+  q.workspace = scratch;
+  q.workspace_bytes = REFORM_EVICT_STATIC_BYTES;
+  return reform_evict_topk(&q, stream);
+}
+
 /* ---------------------------------------------------------------- embed */
 
 int reform_embed_append(const reform_embed_params* p, reform_stream_t stream) {
@@ -298,6 +345,7 @@ const char* reform_status_string(int status) {
     case REFORM_ERR_UNSUPPORTED: return "unsupported dtype, head dimension or alignment";
     case REFORM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case REFORM_ERR_CUDA: return "CUDA call failed";
+    case REFORM_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
