@@ -211,23 +211,32 @@ class Pass:
         else:
             fn()
 
-    def run(self, record=False):
+    def step(self, s, record=False):
+        """Recurrence step s: chunk step, embedding append, eviction into the next buffer set."""
         R, w = self.R, self.w
-        for s in range(w.steps):
-            n_cache = 0 if s == 0 else w.budget
-            self._timed(f"chunk_step{s}", lambda: R.chunk_step(
-                self.q[s], self.k[s], self.v[s], self.out, self.score[s], n_cache, w.window,
-                lse=self.lse, flags=self.flags), record)
-            self._timed("embed_append", lambda: R.embed_append(
-                self.bank, s * w.Lc, self.sel, q_state=self.q[s], k_state=self.kc[s],
-                v_state=self.vc[s]), record)
-            self._timed("evict_topk", lambda: R.evict_topk(
-                self.k[s], self.v[s], self.score[s], self.k[s + 1], self.v[s + 1], self.score[s + 1],
-                n_cache + w.Lc, w.budget, w.n_sink, w.n_recent, kept_idx=self.kept), record)
+        n_cache = 0 if s == 0 else w.budget
+        self._timed(f"chunk_step{s}", lambda: R.chunk_step(
+            self.q[s], self.k[s], self.v[s], self.out, self.score[s], n_cache, w.window,
+            lse=self.lse, flags=self.flags), record)
+        self._timed("embed_append", lambda: R.embed_append(
+            self.bank, s * w.Lc, self.sel, q_state=self.q[s], k_state=self.kc[s],
+            v_state=self.vc[s]), record)
+        self._timed("evict_topk", lambda: R.evict_topk(
+            self.k[s], self.v[s], self.score[s], self.k[s + 1], self.v[s + 1], self.score[s + 1],
+            n_cache + w.Lc, w.budget, w.n_sink, w.n_recent, kept_idx=self.kept), record)
+
+    def tail(self, record=False):
+        """Gather phase: retrieval over the bank the steps wrote, then the row gather."""
+        R, w = self.R, self.w
         self._timed("retrieve_topk", lambda: R.retrieve_topk(
             self.bank, self.queries, w.N, w.k, self.idx, scale=w.sim_scale,
             pool_window=w.pool_window, n_keep_head=w.keep_head, n_keep_tail=w.keep_tail), record)
         self._timed("gather", lambda: R.gather(self.hidden, self.idx, self.gathered), record)
+
+    def run(self, record=False):
+        for s in range(self.w.steps):
+            self.step(s, record)
+        self.tail(record)
 
     def breakdown(self):
         agg = {}
@@ -237,13 +246,16 @@ class Pass:
         return agg
 
 
-class HostPass:
+class HostPipeline:
     """The same pass driven from pinned host buffers: every recurrence step's Q/K/V, the query
     embeddings and the gather source cross PCIe inside the timed region, and the gathered rows
-    and their indices are read back."""
+    and their indices are read back.  Copies run on their own stream one step ahead of the
+    kernels, and two device buffer sets alternate between consecutive passes, so a pass's
+    transfers overlap the previous pass's kernels the way a serving loop streams inputs."""
 
-    def __init__(self, p: Pass):
-        self.p = p
+    def __init__(self, passes):
+        self.sets = passes
+        p = passes[0]
         w = p.w
         pin = lambda t: t.cpu().pin_memory()
         self.hq = [pin(x) for x in p.q]
@@ -257,21 +269,42 @@ class HostPass:
             self.hqueries.numel() * self.hqueries.element_size() + \
             self.hhidden.numel() * self.hhidden.element_size()
         self.d2h = self.hout.numel() * self.hout.element_size() + self.hidx.numel() * 4
+        self.copy_stream = torch.cuda.Stream()
+        self.done = [None] * len(passes)
+        self.count = 0
 
     def run(self):
-        p, w = self.p, self.p.w
+        i = self.count % len(self.sets)
+        self.count += 1
+        p, w = self.sets[i], self.sets[i].w
+        main, cs = torch.cuda.current_stream(), self.copy_stream
+        ready = [torch.cuda.Event() for _ in range(w.steps + 1)]
+        with torch.cuda.stream(cs):
+            if self.done[i] is not None:
+                cs.wait_event(self.done[i])          # this buffer set's previous pass has finished
+            else:
+                cs.wait_stream(main)
+            for s in range(w.steps):
+                p.q[s].copy_(self.hq[s], non_blocking=True)
+                p.kc[s].copy_(self.hk[s], non_blocking=True)
+                p.vc[s].copy_(self.hv[s], non_blocking=True)
+                ready[s].record(cs)
+            p.queries.copy_(self.hqueries, non_blocking=True)
+            p.hidden.copy_(self.hhidden, non_blocking=True)
+            ready[w.steps].record(cs)
+        R = p.R
         for s in range(w.steps):
             n_cache = 0 if s == 0 else w.budget
-            p.q[s].copy_(self.hq[s], non_blocking=True)
-            p.kc[s].copy_(self.hk[s], non_blocking=True)
-            p.vc[s].copy_(self.hv[s], non_blocking=True)
+            main.wait_event(ready[s])
             p.k[s][:, :, n_cache:n_cache + w.Lc].copy_(p.kc[s])
             p.v[s][:, :, n_cache:n_cache + w.Lc].copy_(p.vc[s])
-        p.queries.copy_(self.hqueries, non_blocking=True)
-        p.hidden.copy_(self.hhidden, non_blocking=True)
-        p.run()
+            p.step(s)
+        main.wait_event(ready[w.steps])
+        p.tail()
         self.hout.copy_(p.gathered, non_blocking=True)
         self.hidx.copy_(p.idx, non_blocking=True)
+        self.done[i] = torch.cuda.Event()
+        self.done[i].record(main)
 
 
 def cpu_baseline(w, sample_rows=8192):
@@ -384,7 +417,8 @@ def main():
     # end-to-end arm: host buffers, copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        hp = HostPass(p)
+        hp = HostPipeline([p, Pass(w, dev, seed_offset=rank, force_simt=args.force_simt)])
+        hp.run()
         hp.run()
         barrier()
         start.record()

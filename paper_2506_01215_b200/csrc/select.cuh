@@ -111,6 +111,20 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* scratc
   return res;
 }
 
+// Histogram increment.  When every participating lane of the warp hits the same bin (constant
+// or heavily tied scores, where same-address atomics would serialise) the warp issues one atomic
+// for all of them; otherwise each lane adds its own.  Every lane of the warp must call this
+// (valid = false to sit out).
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t bin, bool valid) {
+  const unsigned active = __ballot_sync(0xffffffffu, valid);
+  if (valid) {
+    int same;
+    __match_all_sync(active, bin, &same);
+    if (!same) atomicAdd(&hist[bin], 1u);
+    else if ((threadIdx.x & 31) == (unsigned)(__ffs(active) - 1)) atomicAdd(&hist[bin], (uint32_t)__popc(active));
+  }
+}
+
 // Executed by the last block of a histogram pass: walk the bins from the top
 // until the running count reaches `remaining`; fix that digit.
 __device__ void sel_find_bin(SelState* st, const uint32_t* hist, int shift, uint32_t* scratch) {
@@ -193,21 +207,18 @@ sel_hist_kernel(SelArgs a, int pass, const float* __restrict__ ts, float* __rest
     for (int j = 0; j < kSelPerThread; ++j) {
       int i = j * kSelThreads + tid;
       long long g = base + i;
-      if (g < a.n) {
-        float v = fmaxf(cur[i], cur[i + window - len]);
-        dst[g] = v;
-        if (g >= a.lo && g < a.hi) atomicAdd(&hist[float_to_key(v) >> shift], 1u);
-      }
+      const float v = fmaxf(cur[i], cur[i + window - len]);
+      if (g < a.n) dst[g] = v;
+      hist_add(hist, float_to_key(v) >> shift, g >= a.lo && g < a.hi);  // every lane calls; hi <= n
     }
   } else {
     __syncthreads();
     const float* src = a.vals + (long long)seg * a.stride;
     for (int j = 0; j < kSelPerThread; ++j) {
       long long g = base + j * kSelThreads + tid;
-      if (g >= a.lo && g < a.hi) {
-        uint32_t key = float_to_key(src[g]);
-        if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & dmask], 1u);
-      }
+      const bool in = g >= a.lo && g < a.hi;
+      const uint32_t key = in ? float_to_key(src[g]) : 0u;
+      hist_add(hist, (key >> shift) & dmask, in && (key & pmask) == prefix);
     }
   }
   __syncthreads();
@@ -245,9 +256,9 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(SelArgs a) {
       eq += key == thr;
     }
   }
-  uint32_t tot_gt, tot_eq;
-  block_excl_scan(gt, scratch, tot_gt);
-  block_excl_scan(eq, scratch, tot_eq);
+  uint32_t tot;  // both counts are <= kSelTile < 2^16: one scan of (gt | eq << 16) serves both
+  block_excl_scan(gt | (eq << 16), scratch, tot);
+  const uint32_t tot_gt = tot & 0xFFFFu, tot_eq = tot >> 16;
   uint2* cnt = a.blockcnt + (size_t)seg * 2 * a.blocks_per_seg;
   uint2* off = cnt + a.blocks_per_seg;
   if (tid == 0) {
@@ -294,10 +305,10 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(SelArgs a) {
       is_gt = key > thr;
       is_eq = key == thr;
     }
-    uint32_t tg, te;
-    uint32_t pg = block_excl_scan(is_gt, scratch, tg);
-    uint32_t pe = block_excl_scan(is_eq, scratch, te);
-    uint32_t gt_before = run_gt + pg, eq_before = run_eq + pe;
+    uint32_t tt;
+    const uint32_t pp = block_excl_scan(is_gt | (is_eq << 16), scratch, tt);
+    const uint32_t tg = tt & 0xFFFFu, te = tt >> 16;
+    uint32_t gt_before = run_gt + (pp & 0xFFFFu), eq_before = run_eq + (pp >> 16);
     if (is_gt || (is_eq && eq_before < need_eq)) {
       uint32_t pos = a.lo + gt_before + (eq_before < need_eq ? eq_before : need_eq);
       out[pos] = (int32_t)g;
@@ -441,7 +452,7 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
     __syncthreads();
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j)
-      if (cand[j] && (key[j] & pmask) == prefix) atomicAdd(&hist[(key[j] >> shift) & dmask], 1u);
+      hist_add(hist, (key[j] >> shift) & dmask, cand[j] && (key[j] & pmask) == prefix);
     __syncthreads();
     uint32_t* gh = a.hist + ((size_t)seg * 3 + pass) * kSelBins;
     for (int i = tid; i < kSelBins; i += kSelThreads) {
@@ -466,9 +477,9 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
     gt += is_gt[j];
     eq += is_eq[j];
   }
-  uint32_t tot_gt, tot_eq;
-  block_excl_scan(gt, scratch, tot_gt);
-  block_excl_scan(eq, scratch, tot_eq);
+  uint32_t tot;  // both counts are <= kSelTile < 2^16: one scan of (gt | eq << 16) serves both
+  block_excl_scan(gt | (eq << 16), scratch, tot);
+  const uint32_t tot_gt = tot & 0xFFFFu, tot_eq = tot >> 16;
   uint2* cnt = a.blockcnt + (size_t)seg * 2 * a.blocks_per_seg;
   if (tid == 0) cnt[blockIdx.x] = make_uint2(tot_gt, tot_eq);
   if (!sel_seg_barrier(ctl, ++phase * nblk, dev_status)) return;
@@ -486,10 +497,10 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
   int32_t* out = a.out + (long long)seg * a.out_stride;
 #pragma unroll
   for (int j = 0; j < kSelPerThread; ++j) {
-    uint32_t tg, te;
-    uint32_t sg = block_excl_scan(is_gt[j], scratch, tg);
-    uint32_t se = block_excl_scan(is_eq[j], scratch, te);
-    uint32_t gt_before = run_gt + sg, eq_before = run_eq + se;
+    uint32_t tt;
+    const uint32_t pp = block_excl_scan(is_gt[j] | (is_eq[j] << 16), scratch, tt);
+    const uint32_t tg = tt & 0xFFFFu, te = tt >> 16;
+    uint32_t gt_before = run_gt + (pp & 0xFFFFu), eq_before = run_eq + (pp >> 16);
     if (is_gt[j] || (is_eq[j] && eq_before < need_eq)) {
       uint32_t pos = a.lo + gt_before + (eq_before < need_eq ? eq_before : need_eq);
       out[pos] = (int32_t)(base + j * kSelThreads + tid);
@@ -506,6 +517,117 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
 
 // Enqueue the whole selection.  If ts != nullptr the first pass pools ts with
 // the given radius into pooled (which must then be a.vals).
+
+// ---------------------------------------------------------------------------
+// One block per segment, used when a call batches many short segments (cache
+// compression of many layers / sequences / KV heads at once, each up to 64K
+// keys): the whole selection is block-local -- the
+// three digit passes histogram in shared memory, the digit decision is made by
+// the block itself, and the ordered write walks the segment once more with
+// warp ballots (each warp owns a contiguous range, so ranks come from popc on
+// ballot masks and a single scan over the 32 warp totals).  No global atomics,
+// no grid-wide waits, nothing to initialise; segments run in parallel.
+// ---------------------------------------------------------------------------
+constexpr int kSelBlockMaxN = 65536;
+constexpr int kSelBlockUnroll = 8;
+constexpr int kSelBlockMinSegs = 48;  // fewer segments than this: spread each one over several blocks instead
+
+__global__ void __launch_bounds__(kSelThreads) sel_block_kernel(SelArgs a) {
+  __shared__ uint32_t hist[kSelBins];
+  __shared__ uint32_t scratch[33];
+  __shared__ uint32_t result[2];
+  __shared__ uint32_t warp_gt[32], warp_eq[32];
+  const int seg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* src = a.vals + (long long)seg * a.stride;
+  int32_t* out = a.out + (long long)seg * a.out_stride;
+  const int ncand = a.hi - a.lo;
+  uint32_t prefix = 0, remaining = (uint32_t)a.m;
+#pragma unroll 1
+  for (int pass = 0; pass < 3; ++pass) {
+    int shift;
+    uint32_t dmask, pmask;
+    sel_pass_params(pass, shift, dmask, pmask);
+    for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+    __syncthreads();
+    // uniform trip count (every lane calls hist_add); eight independent loads per thread in flight
+    for (int i0 = 0; i0 < ncand; i0 += kSelBlockUnroll * kSelThreads) {
+      uint32_t key[kSelBlockUnroll];
+#pragma unroll
+      for (int u = 0; u < kSelBlockUnroll; ++u) {
+        const int i = i0 + u * kSelThreads + tid;
+        key[u] = (i < ncand) ? float_to_key(__ldg(src + a.lo + i)) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < kSelBlockUnroll; ++u) {
+        const bool in = i0 + u * kSelThreads + tid < ncand;
+        hist_add(hist, (key[u] >> shift) & dmask, in && (key[u] & pmask) == prefix);
+      }
+    }
+    __syncthreads();
+    int b0 = kSelBins - 1 - 2 * tid;
+    uint32_t c0 = hist[b0], c1 = hist[b0 - 1];
+    uint32_t total;
+    uint32_t before = block_excl_scan(c0 + c1, scratch, total);
+    if (tid == 0) { result[0] = kSelBins - 1; result[1] = 0; }
+    __syncthreads();
+    if (before < remaining && remaining <= before + c0 + c1) {
+      if (remaining <= before + c0) { result[0] = b0; result[1] = remaining - before; }
+      else { result[0] = b0 - 1; result[1] = remaining - before - c0; }
+    }
+    __syncthreads();
+    prefix |= result[0] << shift;
+    remaining = result[1];
+    __syncthreads();
+  }
+  const uint32_t thr = prefix, need_eq = remaining;
+  // ordered write: warp w owns candidates [w * per_warp, (w + 1) * per_warp)
+  constexpr int kStep = 32 * kSelBlockUnroll;
+  const int per_warp = ((ncand + 31) / 32 + kStep - 1) / kStep * kStep;  // multiple of 32 * unroll
+  const int w0 = warp * per_warp;
+  uint32_t gt = 0, eq = 0;
+  for (int i0 = 0; i0 < per_warp; i0 += kStep) {
+    uint32_t key[kSelBlockUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelBlockUnroll; ++u) {
+      const int i = w0 + i0 + 32 * u + lane;
+      key[u] = (i < ncand) ? float_to_key(__ldg(src + a.lo + i)) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kSelBlockUnroll; ++u) {
+      const bool in = w0 + i0 + 32 * u + lane < ncand;
+      gt += __popc(__ballot_sync(0xffffffffu, in && key[u] > thr));
+      eq += __popc(__ballot_sync(0xffffffffu, in && key[u] == thr));
+    }
+  }
+  if (lane == 0) { warp_gt[warp] = gt; warp_eq[warp] = eq; }
+  __syncthreads();
+  uint32_t run_gt = 0, run_eq = 0;
+  for (int ww = 0; ww < warp; ++ww) { run_gt += warp_gt[ww]; run_eq += warp_eq[ww]; }
+  const uint32_t below = (1u << lane) - 1u;
+  for (int i0 = 0; i0 < per_warp; i0 += kStep) {
+    uint32_t key[kSelBlockUnroll];
+#pragma unroll
+    for (int u = 0; u < kSelBlockUnroll; ++u) {
+      const int i = w0 + i0 + 32 * u + lane;
+      key[u] = (i < ncand) ? float_to_key(__ldg(src + a.lo + i)) : 0u;
+    }
+#pragma unroll
+    for (int u = 0; u < kSelBlockUnroll; ++u) {
+      const int i = w0 + i0 + 32 * u + lane;
+      const bool is_gt = i < ncand && key[u] > thr, is_eq = i < ncand && key[u] == thr;
+      const unsigned mg = __ballot_sync(0xffffffffu, is_gt), me = __ballot_sync(0xffffffffu, is_eq);
+      const uint32_t gt_before = run_gt + __popc(mg & below), eq_before = run_eq + __popc(me & below);
+      if (is_gt || (is_eq && eq_before < need_eq))
+        out[a.lo + gt_before + (eq_before < need_eq ? eq_before : need_eq)] = a.lo + i;
+      run_gt += __popc(mg);
+      run_eq += __popc(me);
+    }
+  }
+  for (int i = tid; i < a.lo; i += kSelThreads) out[i] = i;
+  const int tail = a.n - a.hi;
+  for (int i = tid; i < tail; i += kSelThreads) out[a.lo + a.m + i] = a.hi + i;
+}
+
 // Blocks of sel_fused_kernel that can be resident at once on this device (0 if unknown).
 template <bool POOL>
 inline int sel_fused_capacity(size_t smem) {
@@ -521,6 +643,11 @@ inline int sel_fused_capacity(size_t smem) {
 inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, int radius,
                          void* ws_base, const SelLayout& L, int32_t* dev_status, cudaStream_t st) {
   if (segs == 0) return REFORM_OK;
+  if (!ts && a.n <= kSelBlockMaxN && segs >= kSelBlockMinSegs) {
+    sel_block_kernel<<<segs, kSelThreads, 0, st>>>(a);
+    count_launch();
+    return check_launch();
+  }
   dim3 grid(a.blocks_per_seg, segs);
   {
     const size_t smem = ts ? sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius) : 0;

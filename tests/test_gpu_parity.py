@@ -144,9 +144,8 @@ def test_evict_matches_oracle_bit_exactly(B, Hkv, d, n_keys, budget, sink, recen
     assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept])
 
 
-def test_evict_many_segments_multi_launch_path():
-    """More blocks than can be resident at once: the selection falls back to
-    one launch per pass; results must not change."""
+def test_evict_many_segments():
+    """384 segments in one call (layers x sequences x KV heads batched): one block per segment."""
     g = torch.Generator().manual_seed(4)
     B, Hkv, n, d, budget = 48, 8, 4200, 4, 1000
     k = torch.randn(B, Hkv, n, d, generator=g)
@@ -159,6 +158,39 @@ def test_evict_many_segments_multi_launch_path():
     R.evict_topk(k.to(DEV), k.to(DEV).clone(), sc.to(DEV), kd, vd, sd, n, budget, 16, 16, kept_idx=kept)
     assert torch.equal(kept.cpu(), ref["kept_idx"])
     assert torch.equal(kd.cpu(), ref["k"])
+
+
+def test_evict_long_segments_cooperative_path():
+    """Segments longer than one block handles alone: the selection runs as one cooperative launch."""
+    g = torch.Generator().manual_seed(8)
+    B, Hkv, n, d, budget = 1, 2, 70001, 4, 9000
+    k = torch.randn(B, Hkv, n, d, generator=g)
+    sc = (torch.rand(B, Hkv, n, generator=g) * 4000).floor()
+    ref = oracle.evict_topk(k, k, sc, n, budget, 100, 100, cap_dst=budget)
+    kd = torch.zeros(B, Hkv, budget, d, device=DEV)
+    vd = torch.zeros_like(kd)
+    sd = torch.zeros(B, Hkv, budget, device=DEV)
+    kept = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV)
+    R.evict_topk(k.to(DEV), k.to(DEV).clone(), sc.to(DEV), kd, vd, sd, n, budget, 100, 100, kept_idx=kept)
+    assert torch.equal(kept.cpu(), ref["kept_idx"])
+    assert torch.equal(kd.cpu(), ref["k"])
+
+
+def test_retrieve_many_sequences_multi_launch_path():
+    """More selection blocks than can be resident at once: the selection falls back to one launch
+    per pass; results must not change."""
+    g = torch.Generator().manual_seed(6)
+    B, N, E, nq, k = 90, 17000, 32, 2, 500
+    bank = torch.randn(B, N, E, generator=g).bfloat16()
+    qs = torch.randn(B, nq, E, generator=g).bfloat16()
+    ref = oracle.retrieve_topk(bank, qs, N, k, scale=0.25, pool_window=9, n_keep_head=3, n_keep_tail=5)
+    idx = torch.full((B, k), -1, dtype=torch.int32, device=DEV)
+    pooled = torch.zeros(B, N, device=DEV)
+    R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx, scale=0.25, pool_window=9, n_keep_head=3,
+                    n_keep_tail=5, pooled_score_out=pooled)
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    for b in range(B):
+        assert_index_sets_match(idx[b].cpu(), ref["idx"][b], ref["pooled"][b])
 
 
 def test_evict_without_optional_outputs():
