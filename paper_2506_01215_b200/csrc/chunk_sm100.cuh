@@ -268,6 +268,10 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 // registers; the MMA issuer alternates between the tiles, so one tile's
 // softmax hides behind the other tile's two MMAs.
 // ---------------------------------------------------------------------------
+#ifndef REFORM_POLY_EVERY
+#define REFORM_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = REFORM_POLY_EVERY;  // one pair in kPolyEvery takes the polynomial exp2 (0 = none)
 constexpr int kAttn2Threads = 384;  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
 constexpr size_t kAttn2SmemBytes = 6 * kTileBytes + 1024 + 512;
 
@@ -309,9 +313,9 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   uint64_t* v_full = bars + 5;    // [2]
   uint64_t* v_empty = bars + 7;   // [2]
   uint64_t* s_full = bars + 9;    // [2] per tile
-  uint64_t* p_ready = bars + 11;  // [2] per tile
-  uint64_t* o_full = bars + 13;   // [2] per tile
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
+  uint64_t* p_ready = bars + 11;  // [2 tiles][2 halves of the key tile]
+  uint64_t* o_full = bars + 15;   // [2] per tile
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -332,7 +336,8 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       ptx::mbar_init(v_full + s, 1);
       ptx::mbar_init(v_empty + s, 1);
       ptx::mbar_init(s_full + s, 1);
-      ptx::mbar_init(p_ready + s, 128);
+      ptx::mbar_init(p_ready + 2 * s, 128);
+      ptx::mbar_init(p_ready + 2 * s + 1, 128);
       ptx::mbar_init(o_full + s, 1);
     }
     *abort_flag = 0;
@@ -405,9 +410,15 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!ptx::mbar_wait(v_full + s, ph, abort_flag)) break;
         ptx::tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int k = 0; k < 4; ++k)
           ptx::mma_ts(tO0, tS0 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
                       idesc_pv, (j > 0) || (k > 0));
+        if (!ptx::mbar_wait(p_ready + 1, j & 1, abort_flag)) break;
+        ptx::tc_fence_after();
+#pragma unroll
+        for (int k = 4; k < 8; ++k)
+          ptx::mma_ts(tO0, tS0 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
+                      idesc_pv, 1);
         if (j + 1 < n_kt0) {
           if (!ptx::mbar_wait(k_full + s1, ph1, abort_flag)) break;
           ptx::tc_fence_after();
@@ -418,12 +429,18 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         // tile 1
         if (j < n_kt1) {
-          if (!ptx::mbar_wait(p_ready + 1, j & 1, abort_flag)) break;
+          if (!ptx::mbar_wait(p_ready + 2, j & 1, abort_flag)) break;
           ptx::tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
+          for (int k = 0; k < 4; ++k)
             ptx::mma_ts(tO1, tS1 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
                         idesc_pv, (j > 0) || (k > 0));
+          if (!ptx::mbar_wait(p_ready + 3, j & 1, abort_flag)) break;
+          ptx::tc_fence_after();
+#pragma unroll
+          for (int k = 4; k < 8; ++k)
+            ptx::mma_ts(tO1, tS1 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
+                        idesc_pv, 1);
         }
         ptx::mma_commit(v_empty + s);
         if (j + 1 < n_kt1) {
@@ -459,13 +476,18 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         for (int i = 0; i < 128; ++i)
           if (i > thr) v[i] = 0xff800000u;        // -inf
       }
-      float mx0 = __uint_as_float(v[0]), mx1 = __uint_as_float(v[1]);
+      float mx[8];  // eight independent chains of 3-input maxima
 #pragma unroll
-      for (int i = 2; i < 128; i += 4) {
-        mx0 = ptx::max3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-        if (i + 3 < 128) mx1 = ptx::max3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+      for (int c = 0; c < 8; ++c) mx[c] = ptx::max3(__uint_as_float(v[c]), __uint_as_float(v[c + 8]), __uint_as_float(v[c + 16]));
+#pragma unroll
+      for (int i = 24; i < 120; i += 16) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) mx[c] = ptx::max3(mx[c], __uint_as_float(v[i + c]), __uint_as_float(v[i + c + 8]));
       }
-      const float m_new = fmaxf(m, fmaxf(mx0, mx1) * scale_log2);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) mx[c] = fmaxf(mx[c], __uint_as_float(v[120 + c]));
+      const float mxa = ptx::max3(mx[0], mx[1], mx[2]), mxb = ptx::max3(mx[3], mx[4], mx[5]);
+      const float m_new = fmaxf(m, ptx::max3(mxa, mxb, fmaxf(mx[6], mx[7])) * scale_log2);
       if (j == 0) {
         m = m_new;  // key 0 is visible to every row, so m is finite from here on
       } else {
@@ -487,19 +509,33 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       }
       const float neg_m = -m;
-      uint32_t pk[64];
+      // P goes back to TMEM in two halves (keys 0-63, 64-127), each signalled on its own barrier,
+      // so the first four PV MMAs start while the second half is still being exponentiated
 #pragma unroll
-      for (int i = 0; i < 128; i += 2) {
-        float x0, x1;
-        ptx::fma2(x0, x1, __uint_as_float(v[i]), __uint_as_float(v[i + 1]), scale_log2, neg_m);
-        const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);  // ex2(-inf) = 0 for masked columns
-        ptx::add2(l0, l1, p0, p1);
-        pk[i >> 1] = ptx::pack_bf16(p0, p1);
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[32];
+        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;  // two independent pairs of partial row sums
+#pragma unroll
+        for (int i = 0; i < 64; i += 2) {
+          const int e = 64 * half + i;
+          float x0, x1, p0, p1;
+          ptx::fma2(x0, x1, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), scale_log2, neg_m);
+          if (kPolyEvery > 0 && ((e >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1) {
+            ptx::ex2_poly2(p0, p1, x0, x1);  // this share of the exponentials runs on the FMA pipe
+          } else {
+            p0 = ptx::ex2(x0);               // ex2(-inf) = 0 for masked columns
+            p1 = ptx::ex2(x1);
+          }
+          if (i & 2) ptx::add2(b0, b1, p0, p1); else ptx::add2(a0, a1, p0, p1);
+          pk[i >> 1] = ptx::pack_bf16(p0, p1);
+        }
+        ptx::add2(a0, a1, b0, b1);
+        ptx::add2(l0, l1, a0, a1);
+        ptx::tmem_st32(tS + 32 * half, pk);
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(p_ready + 2 * t + half);
       }
-      ptx::tmem_st64(tS, pk);
-      ptx::tmem_st_wait();
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(p_ready + t);
     }
     if (ok && ptx::mbar_wait(o_full + t, 0, abort_flag)) {
       ptx::tc_fence_after();
