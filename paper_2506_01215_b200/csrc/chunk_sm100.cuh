@@ -1,26 +1,27 @@
 // Tensor-core chunk step for bf16, head dimension 128 (sm_100a: tcgen05 MMA
 // with TMEM accumulators, operands staged by TMA with 128-byte swizzle).
 //
-//   attn_sm100_kernel   Sec. 3.1 chunk forward.  One block owns a 128-row query
-//     tile of one head and walks the visible keys [cache ; chunk prefix] in
-//     128-key tiles:  S = Q K^T (SS MMA, fp32 in TMEM) -> online softmax by 128
-//     threads, one query row each, straight out of TMEM -> P (bf16) written
-//     back into the TMEM columns S occupied -> O += P V (A operand from TMEM, V
-//     from shared memory, MN-major).  O stays in TMEM for the whole walk and is
-//     rescaled only when a row maximum grows by more than 2^8.  Two blocks are
-//     resident per SM (256 TMEM columns, 96 KB of shared memory each): while
-//     one block's softmax runs, the other block's MMAs keep the tensor pipe busy.
+//   attn2_sm100_kernel  Sec. 3.1 chunk forward.  One block per SM owns two
+//     128-row query tiles and walks the visible keys [cache ; chunk prefix] in
+//     128-key tiles that both query tiles share:  S = Q K^T (SS MMA, fp32 in
+//     TMEM) -> online softmax by 128 threads per tile, one query row each,
+//     straight out of TMEM -> P (bf16) written back into the TMEM columns S
+//     occupied -> O += P V (A operand from TMEM, V from shared memory,
+//     MN-major).  O stays in TMEM for the whole walk and is rescaled only when
+//     a row maximum grows by more than 2^8.  While one tile's softmax runs, the
+//     other tile's MMAs keep the tensor pipe busy.  Details at the kernel.
 //
 //   score_sm100_kernel  H2O eviction score (Sec. 3.1; Sec. 4 "Common setup").
 //     Key-stationary second pass: a block owns 128 keys (TMEM lanes) of one KV
 //     head and revisits the trailing score_window query rows of the group's G
 //     query heads: S^T = K Q^T, p = exp2(s*c - lse), summed along the queries
 //     by the thread that owns the key.  One owner per key: no atomics, and the
-//     result does not depend on scheduling.
+//     result does not depend on scheduling.  Roles per block (192 threads):
+//     warp 0 = TMA producer (one lane), warp 1 = MMA issuer (one lane) and
+//     TMEM owner, warps 2..5 = 128 epilogue threads (TMEM lane = 32 * (warp %
+//     4) + lane).
 //
-// Roles per block (192 threads): warp 0 = TMA producer (one lane), warp 1 =
-// MMA issuer (one lane) and TMEM owner, warps 2..5 = 128 softmax/epilogue
-// threads (TMEM lane = 32 * (warp % 4) + lane).  All waits are bounded.
+// All waits are bounded.
 #pragma once
 
 #include "common.cuh"
@@ -36,7 +37,6 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;  // one TMA box: 128 rows x 64 c
 constexpr uint32_t kTmemCols = 256;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
-constexpr size_t kAttnSmemBytes = 3 * kTileBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 constexpr size_t kScoreSmemBytes = 3 * kTileBytes + 1024 + 256 + 2 * kT * sizeof(float);
 
 __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
@@ -54,210 +54,6 @@ __device__ __forceinline__ void issue_kmajor_128x128x128(uint32_t d_tmem, uint32
   }
 }
 
-__global__ void __launch_bounds__(kSm100Threads, 2)
-attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ out,
-                  float* __restrict__ lse, int Hq, int Hkv, int Lc, int n_cache, float scale_log2,
-                  int32_t* dev_status) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = align_1024(smem_raw);
-  uint8_t* sQ = smem;
-  uint8_t* sK = smem + kTileBytes;
-  uint8_t* sV = smem + 2 * kTileBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 3 * kTileBytes);
-  uint64_t* q_full = bars + 0;
-  uint64_t* k_full = bars + 1;
-  uint64_t* k_empty = bars + 2;
-  uint64_t* v_full = bars + 3;
-  uint64_t* v_empty = bars + 4;
-  uint64_t* s_full = bars + 5;
-  uint64_t* p_ready = bars + 6;
-  uint64_t* o_full = bars + 7;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_qt = (Lc + kT - 1) / kT;
-  const int qt = n_qt - 1 - (int)blockIdx.x;  // longest tiles first
-  const int h = blockIdx.y % Hq, b = blockIdx.y / Hq;
-  const int g = h / (Hq / Hkv);
-  const int row0 = qt * kT;
-  const int last_row = min(row0 + kT - 1, Lc - 1);
-  const int n_kt = (n_cache + last_row + 1 + kT - 1) / kT;  // key tiles with at least one visible key
-
-  if (threadIdx.x == 0) {
-    ptx::mbar_init(q_full, 1);
-    ptx::mbar_init(k_full, 1);
-    ptx::mbar_init(k_empty, 1);
-    ptx::mbar_init(v_full, 1);
-    ptx::mbar_init(v_empty, 1);
-    ptx::mbar_init(s_full, 1);
-    ptx::mbar_init(p_ready, 128);
-    ptx::mbar_init(o_full, 1);
-    *abort_flag = 0;
-    ptx::fence_barrier_init();
-  }
-  if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, kTmemCols);
-    ptx::tmem_relinquish();
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  ptx::tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base;        // columns [0, 128): S (fp32), later P (bf16, columns [0, 64))
-  const uint32_t tO = tmem_base + kT;   // columns [128, 256): O (fp32)
-
-  if (warp == 0) {
-    if (lane == 0) {
-      ptx::prefetch_tmap(&tmQ);
-      ptx::prefetch_tmap(&tmK);
-      ptx::prefetch_tmap(&tmV);
-      ptx::mbar_expect_tx(q_full, kTileBytes);
-      ptx::tma_load_3d(sQ, &tmQ, q_full, 0, row0, b * Hq + h);
-      ptx::tma_load_3d(sQ + kHalfBytes, &tmQ, q_full, 64, row0, b * Hq + h);
-      int issued_k = 0, issued_v = 0;
-      for (int j = 0; j < n_kt; ++j) {
-        if (!ptx::mbar_wait(k_empty, (j & 1) ^ 1, abort_flag)) break;
-        ptx::mbar_expect_tx(k_full, kTileBytes);
-        ptx::tma_load_3d(sK, &tmK, k_full, 0, j * kT, b * Hkv + g);
-        ptx::tma_load_3d(sK + kHalfBytes, &tmK, k_full, 64, j * kT, b * Hkv + g);
-        issued_k = j + 1;
-        if (!ptx::mbar_wait(v_empty, (j & 1) ^ 1, abort_flag)) break;
-        ptx::mbar_expect_tx(v_full, kTileBytes);
-        ptx::tma_load_3d(sV, &tmV, v_full, 0, j * kT, b * Hkv + g);
-        ptx::tma_load_3d(sV + kHalfBytes, &tmV, v_full, 64, j * kT, b * Hkv + g);
-        issued_v = j + 1;
-      }
-      if (*abort_flag) {  // let copies in flight land before the block's shared memory is released
-        volatile int ignore = 0;
-        ptx::mbar_wait(q_full, 0, &ignore);
-        if (issued_k) ptx::mbar_wait(k_full, (issued_k - 1) & 1, &ignore);
-        if (issued_v) ptx::mbar_wait(v_full, (issued_v - 1) & 1, &ignore);
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc_pv = ptx::idesc_bf16(kT, kT, false, true);  // V is MN-major
-      const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK), aV = ptx::smem_u32(sV);
-      bool ok = ptx::mbar_wait(q_full, 0, abort_flag);
-      for (int j = 0; ok && j < n_kt; ++j) {
-        if (!ptx::mbar_wait(k_full, j & 1, abort_flag)) break;
-        ptx::tc_fence_after();
-        issue_kmajor_128x128x128(tS, aQ, aK);
-        ptx::mma_commit(s_full);
-        ptx::mma_commit(k_empty);
-        if (!ptx::mbar_wait(p_ready, j & 1, abort_flag)) break;
-        if (!ptx::mbar_wait(v_full, j & 1, abort_flag)) break;
-        ptx::tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          // A: P columns [8k, 8k+8) = keys [16k, 16k+16); B: V rows [16k, 16k+16), both 64-column halves
-          ptx::mma_ts(tO, tS + 8 * k, ptx::smem_desc_sw128(aV + k * 2048, kHalfBytes, 1024), idesc_pv,
-                      (j > 0) || (k > 0));
-        }
-        ptx::mma_commit(v_empty);
-        if (j == n_kt - 1) ptx::mma_commit(o_full);
-      }
-    }
-  } else {
-    const int sub = warp & 3;                     // TMEM sub-partition of this warp
-    const int r = 32 * sub + lane;                // row of the tile = TMEM lane
-    const uint32_t lane_addr = (uint32_t)(32 * sub) << 16;
-    const int row = row0 + r;
-    const int lim = n_cache + row;                // last visible key of this row
-    float m = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < n_kt; ++j) {
-      if (!ptx::mbar_wait(s_full, j & 1, abort_flag)) { ok = false; break; }
-      ptx::tc_fence_after();
-      const int key0 = j * kT;
-      const bool need_mask = key0 + kT - 1 > n_cache + row0;
-      uint32_t v[32];
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        ptx::tmem_ld32(tS + lane_addr + 32 * c, v);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float x = __uint_as_float(v[i]);
-          if (need_mask && key0 + 32 * c + i > lim) x = -INFINITY;
-          mx = fmaxf(mx, x);
-        }
-      }
-      const float m_new = fmaxf(m, mx * scale_log2);
-      if (j == 0) {
-        m = m_new;  // key 0 is visible to every row, so m is finite from here on
-      } else {
-        const bool grow = m_new > m + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, grow)) {
-          const float alpha = grow ? ptx::ex2(m - m_new) : 1.0f;
-          if (grow) m = m_new;
-          l *= alpha;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            ptx::tmem_ld32(tO + lane_addr + 32 * c, v);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-            ptx::tmem_st32(tO + lane_addr + 32 * c, v);
-          }
-          ptx::tmem_st_wait();
-        }
-      }
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        ptx::tmem_ld32(tS + lane_addr + 32 * c, v);
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float p0 = ptx::ex2(fmaf(__uint_as_float(v[i]), scale_log2, -m));
-          float p1 = ptx::ex2(fmaf(__uint_as_float(v[i + 1]), scale_log2, -m));
-          if (need_mask) {
-            if (key0 + 32 * c + i > lim) p0 = 0.f;
-            if (key0 + 32 * c + i + 1 > lim) p1 = 0.f;
-          }
-          l += p0 + p1;
-          pk[i >> 1] = ptx::pack_bf16(p0, p1);
-        }
-        ptx::tmem_st16(tS + lane_addr + 16 * c, pk);
-      }
-      ptx::tmem_st_wait();
-      ptx::tc_fence_before();
-      ptx::mbar_arrive(p_ready);
-    }
-    if (ok && ptx::mbar_wait(o_full, 0, abort_flag)) {
-      ptx::tc_fence_after();
-      const float inv = 1.0f / l;
-      __nv_bfloat16* op = out + (((long long)b * Hq + h) * Lc + row) * kT;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        ptx::tmem_ld32(tO + lane_addr + 32 * c, v);
-        if (row < Lc) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 o;
-            o.x = ptx::pack_bf16(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
-            o.y = ptx::pack_bf16(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
-            o.z = ptx::pack_bf16(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
-            o.w = ptx::pack_bf16(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
-            *reinterpret_cast<uint4*>(op + 32 * c + i) = o;
-          }
-        }
-      }
-      if (row < Lc) lse[((long long)b * Hq + h) * Lc + row] = (m + log2f(l)) * kLn2;
-    }
-  }
-  ptx::tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
-  }
-  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
-}
-
-
 // ---------------------------------------------------------------------------
 // Two query tiles per block, one block per SM.  The two tiles (normally the
 // same 128 query rows of two query heads of one KV group, so their walks are
@@ -268,11 +64,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 // registers; the MMA issuer alternates between the tiles, so one tile's
 // softmax hides behind the other tile's two MMAs.
 // ---------------------------------------------------------------------------
-#ifndef REFORM_POLY_EVERY
-#define REFORM_POLY_EVERY 0
-#endif
-constexpr int kPolyEvery = REFORM_POLY_EVERY;  // one pair in kPolyEvery takes the polynomial exp2 (0 = none)
-constexpr int kAttn2Threads = 384;  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
+constexpr int kAttn2Threads = 384;
+// setmaxnreg only redistributes the registers the block was launched with (what one warpgroup gives
+// up is all the others can take; an increase that cannot be met blocks forever), so the split is
+// checked here against the launch allocation and again, at run time, against the compiled kernel.
+constexpr int kAttn2LaunchRegs = 168, kAttn2SoftmaxRegs = 224, kAttn2OtherRegs = 56;
+static_assert(256 * kAttn2SoftmaxRegs + 128 * kAttn2OtherRegs <= kAttn2Threads * kAttn2LaunchRegs,
+              "setmaxnreg split exceeds the block's launch allocation");  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
 constexpr size_t kAttn2SmemBytes = 6 * kTileBytes + 1024 + 512;
 
 struct Attn2Tile {
@@ -353,7 +151,7 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp >= 8) {
-    ptx::setmaxnreg_dec<56>();
+    ptx::setmaxnreg_dec<kAttn2OtherRegs>();
     if (warp == 8 && lane == 0) {
       ptx::prefetch_tmap(&tmQ);
       ptx::prefetch_tmap(&tmK);
@@ -453,7 +251,7 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
   } else {
-    ptx::setmaxnreg_inc<224>();
+    ptx::setmaxnreg_inc<kAttn2SoftmaxRegs>();
     const int t = warp >> 2;                      // which tile this warpgroup serves
     const Attn2Tile tile = t ? t1 : t0;
     const int sub = warp & 3;                     // TMEM sub-partition of this warp
@@ -518,14 +316,9 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
         for (int i = 0; i < 64; i += 2) {
           const int e = 64 * half + i;
-          float x0, x1, p0, p1;
+          float x0, x1;
           ptx::fma2(x0, x1, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), scale_log2, neg_m);
-          if (kPolyEvery > 0 && ((e >> 1) % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1) {
-            ptx::ex2_poly2(p0, p1, x0, x1);  // this share of the exponentials runs on the FMA pipe
-          } else {
-            p0 = ptx::ex2(x0);               // ex2(-inf) = 0 for masked columns
-            p1 = ptx::ex2(x1);
-          }
+          const float p0 = ptx::ex2(x0), p1 = ptx::ex2(x1);  // ex2(-inf) = 0 for masked columns
           if (i & 2) ptx::add2(b0, b1, p0, p1); else ptx::add2(a0, a1, p0, p1);
           pk[i >> 1] = ptx::pack_bf16(p0, p1);
         }
@@ -569,6 +362,7 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   }
   if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
 }
+
 
 // Enumerates the (query head of the group, 128-row query tile of the window)
 // pairs a key tile has to visit, skipping tiles none of whose rows sees it.
@@ -724,7 +518,19 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
 }
 
+// The setmaxnreg split above assumes the register count the compiler gave the kernel at launch;
+// refuse to launch if it ever differs (an unsatisfiable increase would block forever).
+inline bool attn_launch_regs_ok() {
+  static int ok = -1;
+  if (ok < 0) {
+    cudaFuncAttributes a2;
+    ok = cudaFuncGetAttributes(&a2, attn2_sm100_kernel) == cudaSuccess && a2.numRegs == kAttn2LaunchRegs;
+  }
+  return ok == 1;
+}
+
 inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float scale, cudaStream_t st) {
+  if (!attn_launch_regs_ok()) return REFORM_ERR_UNSUPPORTED;
   const int n = p->n_cache + p->Lc;
   const float scale_log2 = scale * kLog2e;
   CUtensorMap tmQ, tmK, tmV;
@@ -734,22 +540,13 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
     g_last_cuda_error = (int)cudaErrorInvalidValue;
     return REFORM_ERR_CUDA;
   }
-  int mode = 0;  // bring-up aid: 1 = tensor-core score pass only, 2 = tensor-core attention only
+  int mode = 0;  // debugging aid: 1 = CUDA-core attention + tensor-core score pass, 2 = the reverse
   if (const char* e = getenv("REFORM_SM100_MODE")) mode = atoi(e);
   int rc;
   if (mode == 1) {
     reform_chunk_params q = *p;
     q.flags |= REFORM_NO_SCORE;
     rc = launch_chunk_simt(&q, lse, scale, st);
-    if (rc != REFORM_OK) return rc;
-  } else if (mode == 3) {
-    cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
-    dim3 grid((p->Lc + kT - 1) / kT, p->B * p->Hq);
-    attn_sm100_kernel<<<grid, kSm100Threads, kAttnSmemBytes, st>>>(
-        tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
-        p->dev_status);
-    count_launch();
-    rc = check_launch();
     if (rc != REFORM_OK) return rc;
   } else {
     cudaFuncSetAttribute(attn2_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttn2SmemBytes);

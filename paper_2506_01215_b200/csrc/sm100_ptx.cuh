@@ -208,14 +208,6 @@ __device__ __forceinline__ void tmem_ld128(uint32_t taddr, uint32_t (&r)[128]) {
       : "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t (&r)[64]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64};"
@@ -257,48 +249,6 @@ __device__ __forceinline__ void mul2(float& y0, float& y1, float a) {
       "}\n"
       : "+f"(y0), "+f"(y1)
       : "f"(a));
-}
-
-// 2^x for two values on the FMA pipe instead of the special-function unit: round x to the nearest
-// integer n with the 1.5 * 2^23 trick, evaluate a cubic for 2^(x - n) on [-0.5, 0.5] (max relative
-// error 7.5e-5, far inside bf16 rounding) with packed fp32 FMAs, then add n into the exponent field.
-// Inputs below -126 (including -inf for masked logits) give ~1e-38.
-__device__ __forceinline__ void ex2_poly2(float& y0, float& y1, float x0, float x1) {
-  asm("{\n"
-      ".reg .b32 a0, a1, t0, t1, q0, q1, k;\n"
-      ".reg .b64 x, t, n, f, p, c;\n"
-      "max.f32 a0, %2, 0fC2FC0000;\n"   // -126
-      "max.f32 a1, %3, 0fC2FC0000;\n"
-      "mov.b64 x, {a0, a1};\n"
-      "mov.b32 k, 0f4B400000;\n"        // 1.5 * 2^23
-      "mov.b64 c, {k, k};\n"
-      "add.rn.f32x2 t, x, c;\n"
-      "mov.b32 k, 0fCB400000;\n"
-      "mov.b64 c, {k, k};\n"
-      "add.rn.f32x2 n, t, c;\n"
-      "mov.b32 k, 0fBF800000;\n"        // -1
-      "mov.b64 c, {k, k};\n"
-      "fma.rn.f32x2 f, n, c, x;\n"      // f = x - n
-      "mov.b32 k, 0f3D61FB78;\n"        // 0.05517146
-      "mov.b64 p, {k, k};\n"
-      "mov.b32 k, 0f3E786EFB;\n"        // 0.24261086
-      "mov.b64 c, {k, k};\n"
-      "fma.rn.f32x2 p, p, f, c;\n"
-      "mov.b32 k, 0f3F31798D;\n"        // 0.69326099
-      "mov.b64 c, {k, k};\n"
-      "fma.rn.f32x2 p, p, f, c;\n"
-      "mov.b32 k, 0f3F7FFB4A;\n"        // 0.99992809
-      "mov.b64 c, {k, k};\n"
-      "fma.rn.f32x2 p, p, f, c;\n"
-      "mov.b64 {q0, q1}, p;\n"
-      "mov.b64 {t0, t1}, t;\n"
-      "shl.b32 t0, t0, 23;\n"
-      "shl.b32 t1, t1, 23;\n"
-      "add.s32 %0, q0, t0;\n"
-      "add.s32 %1, q1, t1;\n"
-      "}\n"
-      : "=r"(*reinterpret_cast<uint32_t*>(&y0)), "=r"(*reinterpret_cast<uint32_t*>(&y1))
-      : "f"(x0), "f"(x1));
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
