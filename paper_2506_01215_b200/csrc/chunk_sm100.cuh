@@ -64,13 +64,13 @@ __device__ __forceinline__ void issue_kmajor_128x128x128(uint32_t d_tmem, uint32
 // registers; the MMA issuer alternates between the tiles, so one tile's
 // softmax hides behind the other tile's two MMAs.
 // ---------------------------------------------------------------------------
-constexpr int kAttn2Threads = 384;
+constexpr int kAttn2Threads = 384;  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
 // setmaxnreg only redistributes the registers the block was launched with (what one warpgroup gives
 // up is all the others can take; an increase that cannot be met blocks forever), so the split is
 // checked here against the launch allocation and again, at run time, against the compiled kernel.
 constexpr int kAttn2LaunchRegs = 168, kAttn2SoftmaxRegs = 224, kAttn2OtherRegs = 56;
 static_assert(256 * kAttn2SoftmaxRegs + 128 * kAttn2OtherRegs <= kAttn2Threads * kAttn2LaunchRegs,
-              "setmaxnreg split exceeds the block's launch allocation");  // warps 0-3 / 4-7: softmax of tile 0 / 1; warp 8: TMA; warp 9: MMA
+              "setmaxnreg split exceeds the block's launch allocation");
 constexpr size_t kAttn2SmemBytes = 6 * kTileBytes + 1024 + 512;
 
 struct Attn2Tile {
