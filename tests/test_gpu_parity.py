@@ -81,6 +81,45 @@ def test_chunk_step_flags_and_scale():
     assert_scores_close(score3[:, :, :224], s_ref[:, :, :224], 32 * 2 / 224)
 
 
+def test_recompute_phase_prefill_and_decode_shapes():
+    """The steps right after the gather (Sec. 3.3, on-demand recomputation): a plain causal prefill
+    of the gathered tokens is the chunk step with an empty cache and no score pass, and a decode
+    step is a one-row chunk over the recomputed cache."""
+    q, k, v, carry = _case(1, 8, 2, 128, 777, 0, torch.bfloat16, seed=21)
+    out, lse, score = _run_chunk(q, k, v, carry, 0, 1, flags=R.NO_SCORE)
+    o_ref, l_ref = oracle.attention(q, k, v, 0)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    assert (lse.cpu().double() - l_ref).abs().max() < 2e-3
+    assert torch.equal(score.cpu(), carry)
+    q, k, v, carry = _case(2, 8, 2, 128, 1, 1500, torch.bfloat16, seed=22)
+    out, lse, _ = _run_chunk(q, k, v, carry, 1500, 1, flags=R.NO_SCORE)
+    o_ref, l_ref = oracle.attention(q, k, v, 1500)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    assert (lse.cpu().double() - l_ref).abs().max() < 2e-3
+
+
+def test_alternative_compressors_through_the_same_calls():
+    """Sec. 5.1 ablation: TOVA scores keys with the last query only and does not accumulate
+    (score_window 1, no carry); StreamingLLM keeps only the initial and recent rows (budget =
+    sink + recent).  Both are parameter settings of the same two entry points."""
+    q, k, v, carry = _case(1, 8, 2, 128, 200, 300, torch.bfloat16, seed=23)
+    out, lse, score = _run_chunk(q, k, v, carry, 300, 1, flags=0)
+    s_ref = oracle.key_scores(q, k, 300, 1)
+    assert_scores_close(score[:, :, :500], s_ref[:, :, :500], 1 * 4 / 500)
+    ref = oracle.evict_topk(k, v, s_ref, 500, 128, 4, 4, cap_dst=128)
+    kd = torch.zeros(1, 2, 128, 128, dtype=torch.bfloat16, device=DEV)
+    vd, sd = torch.zeros_like(kd), torch.zeros(1, 2, 128, device=DEV)
+    kept = torch.zeros(1, 2, 128, dtype=torch.int32, device=DEV)
+    R.evict_topk(k.to(DEV), v.to(DEV), score, kd, vd, sd, 500, 128, 4, 4, kept_idx=kept)
+    for h in range(2):
+        assert_index_sets_match(kept[0, h].cpu(), ref["kept_idx"][0, h], s_ref[0, h])
+    kept2 = torch.zeros(1, 2, 48, dtype=torch.int32, device=DEV)
+    kd2 = torch.zeros(1, 2, 48, 128, dtype=torch.bfloat16, device=DEV)
+    R.evict_topk(k.to(DEV), v.to(DEV), score, kd2, torch.zeros_like(kd2), torch.zeros(1, 2, 48, device=DEV),
+                 500, 48, 16, 32, kept_idx=kept2)
+    assert kept2.cpu()[0, 0].tolist() == list(range(16)) + list(range(468, 500))
+
+
 def test_chunk_step_is_deterministic():
     q, k, v, carry = _case(1, 8, 2, 128, 260, 130, torch.bfloat16, seed=9)
     a = _run_chunk(q, k, v, carry, 130, 128)
