@@ -430,6 +430,9 @@ def main():
         ms_e2e = max_over_ranks(ms_e2e, dist, dev) / args.steps
         e2e = {"value": job_throughput(w, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                "h2d_bytes_per_step": hp.h2d, "d2h_bytes_per_step": hp.d2h}
+    dev_err = R.device_error()
+    if dev_err:
+        raise RuntimeError(f"a kernel reported device error bits {dev_err} during the benchmark")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -473,6 +476,7 @@ def main():
                      "peak_source": pk["source"],
                      "flops_counted": "4*Hq*d*visible pairs (QK^T and PV of unmasked pairs only)"},
         "gpu_launches": launches,
+        "device_error_bits": dev_err,
         "clocks": clocks,
     }
     if e2e:

@@ -28,7 +28,8 @@
  *   - dev_status (optional, device int32): a kernel that gives up on a bounded
  *     wait, or meets an out-of-range index, ORs a REFORM_DEV_* bit into it
  *     instead of trapping; the context stays usable.  The caller zeroes and
- *     reads it.
+ *     reads it.  The same bits are also kept in a per-device word inside the
+ *     library (reform_device_error), so a failure is visible without it.
  *   - workspace: scratch device memory, at least reform_*_workspace_size()
  *     bytes, 256-byte aligned, private to the call while it is in flight.
  *   - Return value: REFORM_OK or a negative REFORM_ERR_* code.  On any error
@@ -305,6 +306,11 @@ int reform_gather(const reform_gather_params* p, reform_stream_t stream);
 const char* reform_status_string(int status);
 /* cudaError_t of the last failed CUDA call made by this thread (0 if none). */
 int reform_last_cuda_error(void);
+/* REFORM_DEV_* bits that kernels of this library have raised on the current device since the last
+ * clear (whether or not the failing call was given a dev_status word), or REFORM_ERR_CUDA.  Reads
+ * device memory with a blocking copy: synchronise the streams of interest first.  clear != 0
+ * resets the word. */
+int reform_device_error(int clear);
 /* major * 10000 + minor * 100 + patch */
 int reform_version(void);
 /* Number of kernels this library has launched from the calling process since

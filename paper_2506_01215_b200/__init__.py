@@ -77,7 +77,7 @@ EXPORTS = (
     "reform_chunk_step", "reform_chunk_step_workspace_size", "reform_evict_topk",
     "reform_evict_topk_workspace_size", "reform_evict_topk_static", "reform_embed_append", "reform_retrieve_topk",
     "reform_retrieve_topk_workspace_size", "reform_gather", "reform_status_string",
-    "reform_last_cuda_error", "reform_version", "reform_kernel_launch_count",
+    "reform_last_cuda_error", "reform_device_error", "reform_version", "reform_kernel_launch_count",
 )
 
 _lib = None
@@ -116,10 +116,22 @@ def lib() -> ctypes.CDLL:
         L.reform_status_string.argtypes = [ctypes.c_int]
         L.reform_status_string.restype = ctypes.c_char_p
         L.reform_last_cuda_error.restype = ctypes.c_int
+        L.reform_device_error.argtypes = [ctypes.c_int]
+        L.reform_device_error.restype = ctypes.c_int
         L.reform_version.restype = ctypes.c_int
         L.reform_kernel_launch_count.restype = ctypes.c_longlong
         _lib = L
     return _lib
+
+
+def device_error(clear: bool = True) -> int:
+    """DEV_* bits raised by any kernel of the library on the current device since the last clear
+    (synchronises the device first)."""
+    torch.cuda.synchronize()
+    rc = int(lib().reform_device_error(1 if clear else 0))
+    if rc < 0:
+        raise ReformError("reform_device_error", rc)
+    return rc
 
 
 def kernel_launch_count() -> int:

@@ -360,7 +360,7 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) report_device_error(dev_status, REFORM_DEV_TIMEOUT);
 }
 
 
@@ -515,7 +515,7 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
-  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) report_device_error(dev_status, REFORM_DEV_TIMEOUT);
 }
 
 // The setmaxnreg split above assumes the register count the compiler gave the kernel at launch;

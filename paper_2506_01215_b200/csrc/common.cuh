@@ -24,6 +24,16 @@ inline int check_launch() {
   return REFORM_OK;
 }
 
+// Sticky per-device error word: every kernel that gives up on a bounded wait or skips a bad index
+// ORs its REFORM_DEV_* bit here (and into the caller's dev_status word when one was passed), so a
+// failure is never silent.  Read and cleared through reform_device_error().
+__device__ int32_t g_device_error = 0;
+
+__device__ __forceinline__ void report_device_error(int32_t* dev_status, int32_t bit) {
+  atomicOr(&g_device_error, bit);
+  if (dev_status) atomicOr(dev_status, bit);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -351,6 +351,20 @@ const char* reform_status_string(int status) {
 }
 
 int reform_last_cuda_error(void) { return g_last_cuda_error; }
+
+int reform_device_error(int clear) {
+  int32_t word = 0;
+  cudaError_t e = cudaMemcpyFromSymbol(&word, g_device_error, sizeof(word));
+  if (e == cudaSuccess && clear && word) {
+    const int32_t zero = 0;
+    e = cudaMemcpyToSymbol(g_device_error, &zero, sizeof(zero));
+  }
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return REFORM_ERR_CUDA;
+  }
+  return word;
+}
 int reform_version(void) { return 100; }
 long long reform_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -153,7 +153,7 @@ scan_sm100_kernel(const __grid_constant__ CUtensorMap tmBank, const __grid_const
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, kScanTmemCols);
   }
-  if (threadIdx.x == 0 && *abort_flag && dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) report_device_error(dev_status, REFORM_DEV_TIMEOUT);
 }
 
 // Returns REFORM_ERR_UNSUPPORTED when the shape does not fit this kernel (the caller then uses

@@ -25,7 +25,7 @@ gather_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ id
     long long j = idx[r];
     uint4* d = dst + r * vec;
     if (j < 0 || j >= n_rows) {
-      if (lane == 0 && dev_status) atomicOr(dev_status, REFORM_DEV_BAD_INDEX);
+      if (lane == 0) report_device_error(dev_status, REFORM_DEV_BAD_INDEX);
       for (int c = lane; c < vec; c += LANES) d[c] = make_uint4(0, 0, 0, 0);
       continue;
     }

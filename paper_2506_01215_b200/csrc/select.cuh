@@ -351,7 +351,7 @@ __device__ __forceinline__ bool sel_seg_barrier(SelFusedCtl* ctl, uint32_t expec
     while (atomicAdd(&ctl->arrived, 0u) < expected) {
       if (*reinterpret_cast<volatile uint32_t*>(&ctl->abort) || clock64() - t0 > 400000000LL) {
         atomicExch(&ctl->abort, 1u);
-        if (dev_status) atomicOr(dev_status, REFORM_DEV_TIMEOUT);
+        report_device_error(dev_status, REFORM_DEV_TIMEOUT);
         failed = 1;
         break;
       }

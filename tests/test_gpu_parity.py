@@ -349,6 +349,10 @@ def test_gather_flags_bad_index_without_faulting():
     R.gather(src, idx, dst, dev_status=status)
     torch.cuda.synchronize()
     assert status.item() == R.DEV_BAD_INDEX
+    assert R.device_error() & R.DEV_BAD_INDEX          # also kept by the library itself
+    assert R.device_error() == 0                       # cleared by the read above
+    R.gather(src, idx, dst)                            # no status word passed: still not silent
+    assert R.device_error() == R.DEV_BAD_INDEX
     assert torch.equal(dst[0, 0], src[0, 3]) and torch.equal(dst[0, 3], src[0, 9])
     assert torch.all(dst[0, 1:3] == 0)
 
