@@ -199,10 +199,12 @@ def test_evict_many_segments():
     assert torch.equal(kd.cpu(), ref["k"])
 
 
-def test_evict_long_segments_cooperative_path():
-    """Segments longer than one block handles alone: the selection runs as one cooperative launch."""
+@pytest.mark.parametrize("n", [70001, 140001])
+def test_evict_long_segments(n):
+    """Segments longer than one block handles alone: the selection runs as one cooperative launch
+    over global-memory histograms (18 and 35 blocks per segment)."""
     g = torch.Generator().manual_seed(8)
-    B, Hkv, n, d, budget = 1, 2, 70001, 4, 9000
+    B, Hkv, d, budget = 1, 2, 4, 9000
     k = torch.randn(B, Hkv, n, d, generator=g)
     sc = (torch.rand(B, Hkv, n, generator=g) * 4000).floor()
     ref = oracle.evict_topk(k, k, sc, n, budget, 100, 100, cap_dst=budget)
@@ -216,10 +218,10 @@ def test_evict_long_segments_cooperative_path():
 
 
 def test_retrieve_many_sequences_multi_launch_path():
-    """More selection blocks than can be resident at once: the selection falls back to one launch
-    per pass; results must not change."""
+    """More selection blocks than can be resident at once (10 sequences x 35 blocks): the selection
+    falls back to one launch per pass; results must not change."""
     g = torch.Generator().manual_seed(6)
-    B, N, E, nq, k = 90, 17000, 32, 2, 500
+    B, N, E, nq, k = 10, 140000, 32, 2, 500
     bank = torch.randn(B, N, E, generator=g).bfloat16()
     qs = torch.randn(B, nq, E, generator=g).bfloat16()
     ref = oracle.retrieve_topk(bank, qs, N, k, scale=0.25, pool_window=9, n_keep_head=3, n_keep_tail=5)
