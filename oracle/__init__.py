@@ -170,6 +170,20 @@ def retrieve_topk(bank, queries, N, k, scale=1.0, pool_window=1, n_keep_head=0, 
     return dict(idx=idx[:, :rc].contiguous(), ts=ts, pooled=pooled, n_out=rc)
 
 
+def rope(x, row_begin, rows, pos_begin, base=10000.0, interleaved=False):
+    """Rotary embedding of rows [row_begin, row_begin+rows) of x [B,H,cap,d] at consecutive
+    positions pos_begin, pos_begin+1, ...; returns a new tensor (other rows copied)."""
+    B, H, cap, d = x.shape
+    y = x.clone()
+    rc = _load().oracle_rope(
+        _dt(x), B, H, d, ctypes.c_longlong(cap), ctypes.c_longlong(int(row_begin)),
+        ctypes.c_longlong(int(rows)), ctypes.c_longlong(int(pos_begin)), ctypes.c_double(base),
+        int(bool(interleaved)), _p(x), _p(y))
+    if rc != 0:
+        raise ValueError("oracle_rope: bad arguments")
+    return y
+
+
 def gather(src, idx):
     """src [B,n_rows,D] (any dtype), idx [B,k] int32 -> [B,k,D]."""
     B, n_rows, D = src.shape

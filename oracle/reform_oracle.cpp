@@ -24,6 +24,8 @@
 //                         cosine scan, max over query tokens, max-pool over
 //                         adjacent tokens, top-k with first/last tokens kept.
 //   oracle_gather         Sec. 3.3 / Alg. 1 GatherRelevant: row gather.
+//   oracle_rope           Sec. 3.1 "reassign the position IDs ... consecutive": rotary
+//                         embedding at consecutive positions.
 //
 // Readings of the paper that it does not fix (reduction over the GQA group is
 // a sum, carried scores add, ties go to the lowest index, forced tokens count
@@ -396,6 +398,37 @@ int oracle_retrieve_topk(int dtype, int B, long long N, long long N_cap, int E, 
     std::memcpy(idx_out + (size_t)b * k, sel.data(), sizeof(int32_t) * (size_t)n_out);
   }
   return n_out;
+}
+
+// Rotary position embedding with consecutive position ids (Sec. 3.1: after compression the
+// cache rows are re-assigned consecutive ids, so row r of [cache ; chunk] sits at position
+// pos_begin + (r - row_begin)).  For rows [row_begin, row_begin + rows) of x [B,H,cap,d]:
+// pair (a, b) of a row is rotated by angle pos * base^(-2 i / d), i the pair index:
+//   a' = a cos - b sin,  b' = b cos + a sin
+// with the pair (x[i], x[i + d/2]) if interleaved == 0 ("rotate-half" layout of the Llama /
+// Mistral family) or (x[2i], x[2i+1]) if interleaved != 0.  One rounding to the tensor dtype.
+int oracle_rope(int dtype, int B, int H, int d, long long cap, long long row_begin, long long rows,
+                long long pos_begin, double base, int interleaved, const void* src, void* dst) {
+  if (d % 2 != 0 || row_begin < 0 || rows < 0 || row_begin + rows > cap || base <= 0.0) return -1;
+  const int half = d / 2;
+  size_t tasks = (size_t)B * H * (size_t)rows;
+  parallel_for(tasks, [&](size_t t) {
+    long long r = (long long)(t % (size_t)rows);
+    size_t bh = t / (size_t)rows;
+    size_t off = (bh * (size_t)cap + (size_t)(row_begin + r)) * (size_t)d;
+    double pos = (double)(pos_begin + r);
+    std::vector<double> y(d);
+    for (int i = 0; i < half; ++i) {
+      double ang = pos * std::pow(base, -2.0 * i / d);
+      double c = std::cos(ang), s = std::sin(ang);
+      int ia = interleaved ? 2 * i : i, ib = interleaved ? 2 * i + 1 : i + half;
+      double a = load_elem(src, dtype, off + ia), b = load_elem(src, dtype, off + ib);
+      y[ia] = a * c - b * s;
+      y[ib] = b * c + a * s;
+    }
+    for (int e = 0; e < d; ++e) store_elem(dst, dtype, off + e, y[e]);
+  });
+  return 0;
 }
 
 // dst[b, r, :] = src[b, idx[b, r], :], rows of row_bytes bytes.

@@ -408,3 +408,52 @@ def test_gather_copies_rows_bit_exactly():
         assert torch.equal(out[b].view(torch.int16), src[b, idx[b].long()].view(torch.int16))
     with pytest.raises(ValueError):
         oracle.gather(src, torch.tensor([[30], [0]], dtype=torch.int32))
+
+
+# --------------------------------------------------------------------- rope
+
+def _rope_ref_half(x, pos, base):
+    """Independent statement of the rotate-half convention in torch fp64."""
+    d = x.shape[-1]
+    inv = base ** (-torch.arange(0, d, 2, dtype=torch.float64) / d)
+    ang = pos[:, None].double() * inv[None, :]
+    cos, sin = torch.cat([ang.cos(), ang.cos()], -1), torch.cat([ang.sin(), ang.sin()], -1)
+    x = x.double()
+    rot = torch.cat([-x[..., d // 2:], x[..., :d // 2]], -1)
+    return x * cos + rot * sin
+
+
+def test_rope_matches_rotate_half_and_complex_forms():
+    g = torch.Generator().manual_seed(31)
+    x = torch.randn(2, 3, 20, 16, generator=g)
+    y = oracle.rope(x, 4, 10, 1000)
+    pos = torch.arange(1000, 1010)
+    ref = _rope_ref_half(x[:, :, 4:14], pos, 10000.0)
+    assert torch.allclose(y[:, :, 4:14].double(), ref, atol=2e-7)          # one fp32 rounding
+    assert torch.equal(y[:, :, :4], x[:, :, :4]) and torch.equal(y[:, :, 14:], x[:, :, 14:])
+    # interleaved pairs = multiplication by e^{i pos theta} of the complex view
+    yi = oracle.rope(x, 4, 10, 1000, base=500.0, interleaved=True)
+    inv = 500.0 ** (-torch.arange(0, 16, 2, dtype=torch.float64) / 16)
+    z = torch.view_as_complex(x[:, :, 4:14].double().reshape(2, 3, 10, 8, 2).contiguous())
+    zr = z * torch.polar(torch.ones(10, 8, dtype=torch.float64), pos[:, None].double() * inv[None, :])
+    assert torch.allclose(yi[:, :, 4:14].double(), torch.view_as_real(zr).reshape(2, 3, 10, 16), atol=2e-7)
+
+
+def test_rope_position_zero_is_identity_and_norms_are_kept():
+    g = torch.Generator().manual_seed(32)
+    x = torch.randn(1, 2, 8, 32, generator=g)
+    y = oracle.rope(x, 0, 8, 0)
+    assert torch.equal(y[:, :, 0], x[:, :, 0])
+    assert torch.allclose(y.double().norm(dim=-1), x.double().norm(dim=-1), rtol=1e-6)
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    g = torch.Generator().manual_seed(33)
+    q = torch.randn(1, 1, 1, 64, generator=g).double().float()
+    k = torch.randn(1, 1, 1, 64, generator=g).double().float()
+    dots = []
+    for m, n in [(5, 2), (1005, 1002), (40963, 40960)]:
+        qm, kn = oracle.rope(q, 0, 1, m), oracle.rope(k, 0, 1, n)
+        dots.append((qm.double() * kn.double()).sum().item())
+    assert abs(dots[0] - dots[1]) < 1e-4 and abs(dots[0] - dots[2]) < 1e-4
+    assert abs(dots[0] - (q.double() * k.double()).sum().item()) > 1e-3   # and it is not the unrotated dot
