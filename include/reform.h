@@ -13,6 +13,8 @@
  *   reform_retrieve_topk  cosine scan of the bank against the query
  *                         embeddings, pooling, top-k token selection
  *   reform_gather         copies the selected rows into a contiguous buffer
+ * and, beside the path, reform_rope (rotary embedding at the consecutive
+ * position ids the compression re-assigns).
  *
  * Conventions common to every call
  *   - All tensor pointers are DEVICE pointers unless a field says "host".
@@ -301,6 +303,40 @@ typedef struct reform_gather_params {
 } reform_gather_params;
 
 int reform_gather(const reform_gather_params* p, reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
+ * reform_rope -- Sec. 3.1: "after compression, we reassign the position IDs so
+ * that the tokens in the compressed cache have consecutive position IDs".
+ * The cache therefore keeps un-rotated keys, and a step rotates its operands
+ * with the ids of the moment: cache row r at position r, chunk row i at
+ * n_cache + i (queries likewise).  This call applies the rotary embedding to
+ * rows [row_begin, row_begin + rows) of every (b, head) at consecutive
+ * positions pos_begin, pos_begin + 1, ...:
+ *   angle = pos * theta_base^(-2 i / d)           i = pair index in [0, d/2)
+ *   a' = a cos(angle) - b sin(angle);   b' = b cos(angle) + a sin(angle)
+ * with pair i = (x[i], x[i + d/2]) (interleaved == 0, the rotate-half layout
+ * of the Llama / Mistral family) or (x[2i], x[2i+1]) (interleaved != 0).
+ * Angles are evaluated in fp64, the rotation in fp32, one rounding to dtype.
+ *
+ *   src [B,H,cap,d] in;  dst [B,H,cap,d] out (may be src: in place); rows
+ *   outside the range are not touched.  theta_base 0 means 10000.
+ * d * sizeof(dtype) must be a multiple of 32.
+ * ------------------------------------------------------------------------ */
+typedef struct reform_rope_params {
+  size_t struct_size;
+  int32_t dtype;
+  int32_t B, H, d;
+  int32_t interleaved;
+  int64_t cap;
+  int64_t row_begin, rows;
+  int64_t pos_begin;
+  float theta_base;
+  const void* src;
+  void* dst;
+  int32_t* dev_status;
+} reform_rope_params;
+
+int reform_rope(const reform_rope_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------ */
 const char* reform_status_string(int status);

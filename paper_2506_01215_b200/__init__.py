@@ -73,10 +73,17 @@ class GatherParams(ctypes.Structure):
                 ("row_bytes", _i64), ("src", _vp), ("idx", _vp), ("dst", _vp), ("dev_status", _vp)]
 
 
+class RopeParams(ctypes.Structure):
+    _fields_ = [("struct_size", _sz), ("dtype", _i32), ("B", _i32), ("H", _i32), ("d", _i32),
+                ("interleaved", _i32), ("cap", _i64), ("row_begin", _i64), ("rows", _i64),
+                ("pos_begin", _i64), ("theta_base", _f32), ("src", _vp), ("dst", _vp),
+                ("dev_status", _vp)]
+
+
 EXPORTS = (
     "reform_chunk_step", "reform_chunk_step_workspace_size", "reform_evict_topk",
     "reform_evict_topk_workspace_size", "reform_evict_topk_static", "reform_embed_append", "reform_retrieve_topk",
-    "reform_retrieve_topk_workspace_size", "reform_gather", "reform_status_string",
+    "reform_retrieve_topk_workspace_size", "reform_gather", "reform_rope", "reform_status_string",
     "reform_last_cuda_error", "reform_device_error", "reform_version", "reform_kernel_launch_count",
 )
 
@@ -113,6 +120,8 @@ def lib() -> ctypes.CDLL:
         L.reform_embed_append.restype = ctypes.c_int
         L.reform_gather.argtypes = [ctypes.POINTER(GatherParams), _vp]
         L.reform_gather.restype = ctypes.c_int
+        L.reform_rope.argtypes = [ctypes.POINTER(RopeParams), _vp]
+        L.reform_rope.restype = ctypes.c_int
         L.reform_status_string.argtypes = [ctypes.c_int]
         L.reform_status_string.restype = ctypes.c_char_p
         L.reform_last_cuda_error.restype = ctypes.c_int
@@ -279,6 +288,16 @@ def gather(src, idx, dst, *, dev_status=None, stream=None):
     _check("reform_gather", lib().reform_gather(ctypes.byref(p), _stream(stream)))
 
 
+def rope(src, dst, row_begin: int, rows: int, pos_begin: int, *, theta_base: float = 0.0,
+         interleaved: bool = False, stream=None):
+    """reform_rope: rotary embedding of rows [row_begin, row_begin+rows) of src [B,H,cap,d] at
+    consecutive positions pos_begin, pos_begin+1, ... into dst (may be src)."""
+    B, H, cap, d = src.shape
+    p = RopeParams(ctypes.sizeof(RopeParams), _dtype_code(src), B, H, d, int(bool(interleaved)), cap,
+                   int(row_begin), int(rows), int(pos_begin), float(theta_base), _ptr(src), _ptr(dst), None)
+    _check("reform_rope", lib().reform_rope(ctypes.byref(p), _stream(stream)))
+
+
 # the C entry points' own names, for callers that prefer them
 reform_chunk_step = chunk_step
 reform_evict_topk = evict_topk
@@ -286,3 +305,4 @@ reform_evict_topk_static = evict_topk_static
 reform_embed_append = embed_append
 reform_retrieve_topk = retrieve_topk
 reform_gather = gather
+reform_rope = rope

@@ -6,6 +6,7 @@
 #include "common.cuh"
 #include "rows.cuh"
 #include "embed.cuh"
+#include "rope.cuh"
 #include "select.cuh"
 #include "retrieve.cuh"
 #include "chunk_simt.cuh"
@@ -334,6 +335,25 @@ int reform_gather(const reform_gather_params* p, reform_stream_t stream) {
     return REFORM_ERR_INVALID_ARG;
   return launch_gather((const uint4*)p->src, p->idx, (uint4*)p->dst, p->B, p->k, p->n_rows,
                        p->row_bytes, p->dev_status, reinterpret_cast<cudaStream_t>(stream));
+}
+
+/* ----------------------------------------------------------------- rope */
+
+int reform_rope(const reform_rope_params* p, reform_stream_t stream) {
+  if (!p || p->struct_size != sizeof(reform_rope_params)) return REFORM_ERR_INVALID_ARG;
+  if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
+  if (p->B < 0 || p->H < 0 || p->d <= 0 || p->cap < 0 || p->row_begin < 0 || p->rows < 0 ||
+      p->row_begin + p->rows > p->cap || p->pos_begin < 0 || !(p->theta_base >= 0.f))
+    return REFORM_ERR_INVALID_ARG;
+  if ((p->d * elem_size(p->dtype)) % 32 != 0) return REFORM_ERR_UNSUPPORTED;
+  if (!p->src || !p->dst || !aligned16(p->src) || !aligned16(p->dst)) return REFORM_ERR_INVALID_ARG;
+  const double base = p->theta_base > 0.f ? (double)p->theta_base : 10000.0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  if (p->dtype == REFORM_F32)
+    return launch_rope<float>(p->src, p->dst, p->B * p->H, p->d, p->cap, p->row_begin, p->rows, p->pos_begin,
+                              base, p->interleaved != 0, st);
+  return launch_rope<__nv_bfloat16>(p->src, p->dst, p->B * p->H, p->d, p->cap, p->row_begin, p->rows,
+                                    p->pos_begin, base, p->interleaved != 0, st);
 }
 
 /* ----------------------------------------------------------------- misc */

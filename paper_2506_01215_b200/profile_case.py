@@ -18,7 +18,7 @@ from paper_2506_01215_b200 import synth
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["chunk_step", "evict", "embed", "retrieve", "gather"])
+    ap.add_argument("op", choices=["chunk_step", "evict", "embed", "retrieve", "gather", "rope"])
     ap.add_argument("--workload", default="llama8b_128k")
     ap.add_argument("--lc", type=int, default=8192)
     ap.add_argument("--budget", type=int, default=8192)
@@ -36,7 +36,7 @@ def main():
     w = dataclasses.replace(w, Lc=a.lc, budget=a.budget, window=min(a.window, a.lc), T=2 * a.lc, N=a.n,
                             nq=a.nq or w.nq, k=a.k or w.k)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if a.op in ("chunk_step", "embed", "evict"):
+    if a.op in ("chunk_step", "embed", "evict", "rope"):
         wb = dataclasses.replace(w, B=w.B * a.layers) if a.op == "evict" else w
         q, kc, vc = synth.chunk_qkv(wb, 0, 1, device=dev)
         k0, v0, s0 = synth.cache_state(wb, 0, device=dev)
@@ -57,6 +57,12 @@ def main():
         bank = torch.zeros(w.B, w.Lc, w.E, dtype=w.dtype, device=dev)
         sel = synth.head_selection(w)
         fn = lambda: R.embed_append(bank, 0, sel, q_state=q, k_state=kc, v_state=vc)
+    elif a.op == "rope":
+        q_rot, k_rot = torch.empty_like(q), torch.empty_like(k)
+
+        def fn():
+            R.rope(q, q_rot, 0, w.Lc, w.budget)      # queries at positions n_cache + i
+            R.rope(k, k_rot, 0, w.cap, 0)            # cache and chunk keys at positions 0 .. n-1
     elif a.op == "retrieve":
         bank, queries, _ = synth.bank_and_queries(w, device=dev)
         idx = torch.zeros(w.B, w.k, dtype=torch.int32, device=dev)

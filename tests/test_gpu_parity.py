@@ -430,3 +430,50 @@ def test_tiny_free_running_pipeline_with_driver():
         same = (cache.k[cache.cur][:, :, :n_cache].cpu() == ck[:, :, :n_cache]).all(-1).float().mean().item()
         assert same > 0.995, f"step {step}: only {same:.4f} of cache rows agree"
     assert_scores_close(cache.score[cache.cur][:, :, :n_cache], cs[:, :, :n_cache], 1e-3) if same == 1.0 else None
+
+
+# ------------------------------------------------------------------- rope
+
+@pytest.mark.parametrize("dtype,d,interleaved,pos0", [
+    (torch.bfloat16, 128, False, 0), (torch.bfloat16, 128, False, 1000000), (torch.bfloat16, 64, True, 40960),
+    (torch.float32, 64, False, 8191), (torch.float32, 32, True, 5),
+])
+def test_rope_matches_oracle(dtype, d, interleaved, pos0):
+    g = torch.Generator().manual_seed(d + pos0 % 97)
+    x = torch.randn(2, 3, 150, d, generator=g).to(dtype)
+    ref = oracle.rope(x, 7, 131, pos0, base=500000.0, interleaved=interleaved)
+    xd = x.to(DEV)
+    yd = torch.full_like(xd, 3.0)
+    R.rope(xd, yd, 7, 131, pos0, theta_base=500000.0, interleaved=interleaved)
+    got = yd.cpu()
+    assert torch.all(got[:, :, :7] == 3.0) and torch.all(got[:, :, 138:] == 3.0)   # untouched rows
+    a, b = got[:, :, 7:138].double(), ref[:, :, 7:138].double()
+    # both sides are rounded to dtype: they may land one unit in the last place apart (spacing is
+    # up to 2^-7 of the value in bf16); the fp32 rotation itself is good to a few fp32 ulps
+    ulp = 2.0 ** -7 if dtype == torch.bfloat16 else 2.0 ** -21
+    assert ((a - b).abs() <= ulp * b.abs() + 1e-6).all()
+    if dtype == torch.bfloat16:
+        assert (got[:, :, 7:138] == ref[:, :, 7:138]).float().mean().item() > 0.99
+    R.rope(xd, xd, 7, 131, pos0, theta_base=500000.0, interleaved=interleaved)          # in place
+    assert torch.equal(xd[:, :, 7:138], yd[:, :, 7:138])
+    assert torch.equal(xd.cpu()[:, :, :7], x[:, :, :7])
+
+
+def test_chunk_step_on_rotated_operands():
+    """One recurrence step as a model would run it: un-rotated cache and chunk keys are rotated at
+    the consecutive ids of the moment (cache row r -> r, chunk row i -> n_cache + i), queries at
+    n_cache + i, then the chunk step; against the oracle doing the same in fp64."""
+    q, k, v, carry = _case(1, 8, 2, 128, 200, 300, torch.bfloat16, seed=41)
+    n_cache, n = 300, 500
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    q_rot, k_rot = torch.empty_like(qd), kd.clone()
+    R.rope(qd, q_rot, 0, 200, n_cache)
+    R.rope(kd, k_rot, 0, n, 0)
+    out = torch.empty_like(qd)
+    score = carry.to(DEV).clone()
+    R.chunk_step(q_rot, k_rot, vd, out, score, n_cache, 128, flags=R.SCORE_ACCUMULATE)
+    qo, ko = oracle.rope(q, 0, 200, n_cache), oracle.rope(k, 0, n, 0)
+    o_ref, _ = oracle.attention(qo, ko, v, n_cache)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    s_ref = oracle.key_scores(qo, ko, n_cache, 128, score_in=carry, accumulate=True)
+    assert_scores_close(score[:, :, :n], s_ref[:, :, :n], 128 * 4 / n)

@@ -167,3 +167,19 @@ def test_binding_refuses_host_tensors():
     t = torch.zeros(1, 4, 8)
     with pytest.raises(ValueError):
         R.gather(t, torch.zeros(1, 2, dtype=torch.int32), torch.zeros(1, 2, 8))
+
+
+def _rope(**kw):
+    base = dict(struct_size=ctypes.sizeof(R.RopeParams), dtype=R.BF16, B=1, H=2, d=128, interleaved=0, cap=64,
+                row_begin=0, rows=64, pos_begin=0, theta_base=0.0, src=FAKE, dst=FAKE, dev_status=None)
+    base.update(kw)
+    return R.RopeParams(**base)
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(rows=65), R.ERR_INVALID_ARG), (dict(row_begin=-1), R.ERR_INVALID_ARG), (dict(pos_begin=-5), R.ERR_INVALID_ARG),
+    (dict(src=None), R.ERR_INVALID_ARG), (dict(theta_base=-1.0), R.ERR_INVALID_ARG), (dict(struct_size=4), R.ERR_INVALID_ARG),
+    (dict(d=24), R.ERR_UNSUPPORTED), (dict(dtype=9), R.ERR_UNSUPPORTED),
+])
+def test_rope_rejects_bad_arguments(kw, code):
+    assert R.lib().reform_rope(ctypes.byref(_rope(**kw)), None) == code
