@@ -183,3 +183,27 @@ def _rope(**kw):
 ])
 def test_rope_rejects_bad_arguments(kw, code):
     assert R.lib().reform_rope(ctypes.byref(_rope(**kw)), None) == code
+
+
+def test_empty_inputs_are_accepted_and_launch_nothing():
+    """Degenerate sizes return REFORM_OK before any CUDA call (so this runs without a GPU)."""
+    L = R.lib()
+    n0 = R.kernel_launch_count()
+    assert L.reform_chunk_step(ctypes.byref(_chunk(B=0)), None) == R.OK
+    assert L.reform_chunk_step(ctypes.byref(_chunk(Lc=0, n_cache=0, score_window=0)), None) == R.OK
+    assert L.reform_evict_topk(ctypes.byref(_evict(B=0)), None) == R.OK
+    n = ctypes.c_int32(-1)
+    assert L.reform_evict_topk(ctypes.byref(_evict(n_keys=0, n_kept_host=ctypes.addressof(n))), None) == R.OK
+    assert n.value == 0
+    assert L.reform_evict_topk(ctypes.byref(_evict(budget=0, n_sink=0, n_recent=0)), None) == R.OK
+    p, _keep = _embed(Lc=0)
+    assert L.reform_embed_append(ctypes.byref(p), None) == R.OK
+    p, _keep = _embed(sel=(), n_sel=0)
+    assert L.reform_embed_append(ctypes.byref(p), None) == R.OK
+    assert L.reform_retrieve_topk(ctypes.byref(_retrieve(N=0)), None) == R.OK
+    assert L.reform_retrieve_topk(ctypes.byref(_retrieve(k=0, n_keep_head=0, n_keep_tail=0)), None) == R.OK
+    assert L.reform_retrieve_topk(ctypes.byref(_retrieve(B=0)), None) == R.OK
+    assert L.reform_gather(ctypes.byref(_gather(k=0)), None) == R.OK
+    assert L.reform_gather(ctypes.byref(_gather(B=0)), None) == R.OK
+    assert L.reform_rope(ctypes.byref(_rope(rows=0)), None) == R.OK
+    assert R.kernel_launch_count() == n0
