@@ -97,6 +97,10 @@ enum { REFORM_STATE_Q = 0, REFORM_STATE_K = 1, REFORM_STATE_V = 2 };
  *   score  [B,Hkv,cap]    fp32 in/out; rows [0, n_cache+Lc) are written
  * d is 64 or 128.  dtype REFORM_BF16 with d == 128 runs on the tensor cores
  * (fp32 accumulate); REFORM_F32, and bf16 with d == 64, run on CUDA cores.
+ * Decode-shaped steps (bf16, d == 128, Lc * Hq / Hkv <= 16: a few new tokens
+ * over the recomputed cache) take a split-key kernel that needs workspace for
+ * its partial results even when lse is given: always size the workspace with
+ * reform_chunk_step_workspace_size().
  * softmax_scale 0 means 1/sqrt(d).  score_window in [1, Lc].
  * ------------------------------------------------------------------------ */
 typedef struct reform_chunk_params {

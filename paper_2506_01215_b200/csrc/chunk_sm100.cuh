@@ -529,7 +529,9 @@ inline bool attn_launch_regs_ok() {
   return ok == 1;
 }
 
-inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float scale, cudaStream_t st) {
+// run_attention == false: only the score pass (lse already holds the row normalisers).
+inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float scale, cudaStream_t st,
+                              bool run_attention = true) {
   if (!attn_launch_regs_ok()) return REFORM_ERR_UNSUPPORTED;
   const int n = p->n_cache + p->Lc;
   const float scale_log2 = scale * kLog2e;
@@ -542,8 +544,10 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
   }
   int mode = 0;  // debugging aid: 1 = CUDA-core attention + tensor-core score pass, 2 = the reverse
   if (const char* e = getenv("REFORM_SM100_MODE")) mode = atoi(e);
-  int rc;
-  if (mode == 1) {
+  int rc = REFORM_OK;
+  if (!run_attention) {
+    // nothing to do here
+  } else if (mode == 1) {
     reform_chunk_params q = *p;
     q.flags |= REFORM_NO_SCORE;
     rc = launch_chunk_simt(&q, lse, scale, st);

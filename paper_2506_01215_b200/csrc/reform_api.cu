@@ -15,6 +15,7 @@
 #endif
 #ifndef REFORM_NO_SM100
 #include "chunk_sm100.cuh"
+#include "decode.cuh"
 #include "retrieve_sm100.cuh"
 #endif
 
@@ -29,6 +30,18 @@ static bool dtype_ok(int dtype) { return dtype == REFORM_F32 || dtype == REFORM_
 static size_t chunk_lse_bytes(const reform_chunk_params* p) {
   return align_up(sizeof(float) * (size_t)p->B * p->Hq * p->Lc, 256);
 }
+
+// Decode-shaped steps (a few query rows per KV head) take the split-KV kernel.
+static bool chunk_uses_decode(const reform_chunk_params* p) {
+#ifndef REFORM_NO_SM100
+  return p->Lc > 0 && decode_shape(p) && !(p->flags & REFORM_FORCE_SIMT);
+#else
+  (void)p;
+  return false;
+#endif
+}
+
+static size_t chunk_workspace_bytes(const reform_chunk_params* p);
 
 static bool chunk_uses_sm100(const reform_chunk_params* p) {
 #ifndef REFORM_NO_SM100
@@ -58,6 +71,16 @@ static int validate_chunk(const reform_chunk_params* p) {
 }
 }  // namespace reform
 
+namespace reform {
+static size_t chunk_workspace_bytes(const reform_chunk_params* p) {
+  size_t bytes = p->lse ? 0 : chunk_lse_bytes(p);
+#ifndef REFORM_NO_SM100
+  if (chunk_uses_decode(p)) bytes += decode_workspace_bytes(p);
+#endif
+  return bytes;
+}
+}  // namespace reform
+
 using namespace reform;
 
 extern "C" {
@@ -65,23 +88,30 @@ extern "C" {
 size_t reform_chunk_step_workspace_size(const reform_chunk_params* p) {
   if (!p || p->struct_size != sizeof(reform_chunk_params)) return 0;
   if (p->B <= 0 || p->Hq <= 0 || p->Lc <= 0) return 0;
-  return p->lse ? 0 : chunk_lse_bytes(p);
+  return chunk_workspace_bytes(p);
 }
 
 int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream) {
   int rc = validate_chunk(p);
   if (rc != REFORM_OK) return rc;
-  float* lse = p->lse;
-  if (!lse) {
-    if (!p->workspace || p->workspace_bytes < chunk_lse_bytes(p) ||
-        (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
-      return REFORM_ERR_WORKSPACE;
-    lse = reinterpret_cast<float*>(p->workspace);
-  }
   if (p->B == 0 || p->Lc == 0) return REFORM_OK;
+  float* lse = p->lse;
+  char* ws = reinterpret_cast<char*>(p->workspace);
+  const size_t need = chunk_workspace_bytes(p);
+  if (need && (!ws || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)))
+    return REFORM_ERR_WORKSPACE;
+  if (!lse) {
+    lse = reinterpret_cast<float*>(ws);
+    ws += chunk_lse_bytes(p);
+  }
   float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->d);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 #ifndef REFORM_NO_SM100
+  if (chunk_uses_decode(p)) {
+    rc = launch_decode(p, lse, scale, ws, st);
+    if (rc != REFORM_OK || (p->flags & REFORM_NO_SCORE)) return rc;
+    return launch_chunk_sm100(p, lse, scale, st, /*run_attention=*/false);
+  }
   if (chunk_uses_sm100(p)) return launch_chunk_sm100(p, lse, scale, st);
 #endif
   return launch_chunk_simt(p, lse, scale, st);

@@ -98,6 +98,27 @@ def test_recompute_phase_prefill_and_decode_shapes():
     assert (lse.cpu().double() - l_ref).abs().max() < 2e-3
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,Lc,n_cache,W", [
+    (1, 32, 8, 1, 8192, 1),      # one new token over an 8k recomputed cache (the decode step)
+    (2, 8, 2, 4, 1000, 4),       # four tokens at once: 16 packed rows, causal among themselves
+    (1, 12, 4, 3, 77, 2),        # group of 3, ragged everything
+    (1, 4, 4, 5, 0, 5),          # no sharing, empty cache
+    (1, 16, 1, 1, 300, 1),       # all 16 heads on one KV head
+])
+def test_decode_shaped_steps_match_oracle(B, Hq, Hkv, Lc, n_cache, W):
+    """Few query rows per KV head: the split-KV kernel (keys divided among warps, partials merged)."""
+    q, k, v, carry = _case(B, Hq, Hkv, 128, Lc, n_cache, torch.bfloat16, seed=n_cache + Lc)
+    out, lse, score = _run_chunk(q, k, v, carry, n_cache, W)
+    o_ref, l_ref = oracle.attention(q, k, v, n_cache)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    assert (lse.cpu().double() - l_ref).abs().max() < 2e-3
+    n = n_cache + Lc
+    s_ref = oracle.key_scores(q, k, n_cache, W, score_in=carry, accumulate=True)
+    assert_scores_close(score[:, :, :n], s_ref[:, :, :n], W * (Hq // Hkv) / n)
+    out2, lse2, _ = _run_chunk(q, k, v, carry, n_cache, W, flags=R.FORCE_SIMT | R.SCORE_ACCUMULATE)
+    assert (out2.float() - out.float()).abs().max() < 2e-2
+
+
 def test_alternative_compressors_through_the_same_calls():
     """Sec. 5.1 ablation: TOVA scores keys with the last query only and does not accumulate
     (score_window 1, no carry); StreamingLLM keeps only the initial and recent rows (budget =
