@@ -340,6 +340,12 @@ struct SelFusedCtl {   // per segment, zeroed before the launch
   uint32_t pad[2];
 };
 
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
 __device__ __forceinline__ bool sel_seg_barrier(SelFusedCtl* ctl, uint32_t expected, int32_t* dev_status) {
   __shared__ int failed;
   __syncthreads();
@@ -348,7 +354,7 @@ __device__ __forceinline__ bool sel_seg_barrier(SelFusedCtl* ctl, uint32_t expec
     __threadfence();
     atomicAdd(&ctl->arrived, 1u);
     const long long t0 = clock64();
-    while (atomicAdd(&ctl->arrived, 0u) < expected) {
+    while (ld_acquire_u32(&ctl->arrived) < expected) {  // plain acquire loads: polling with atomics would serialise in L2
       if (*reinterpret_cast<volatile uint32_t*>(&ctl->abort) || clock64() - t0 > 400000000LL) {
         atomicExch(&ctl->abort, 1u);
         report_device_error(dev_status, REFORM_DEV_TIMEOUT);
