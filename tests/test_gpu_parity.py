@@ -338,6 +338,20 @@ def test_retrieve_matches_oracle(name, N, pool, keep, k):
             assert set(planted[b]) <= set(idx[b].tolist())
 
 
+def test_retrieve_window_wider_than_the_bank():
+    g = torch.Generator().manual_seed(12)
+    bank = torch.randn(2, 50, 64, generator=g).bfloat16()
+    qs = torch.randn(2, 3, 64, generator=g).bfloat16()
+    ref = oracle.retrieve_topk(bank, qs, 50, 7, scale=0.5, pool_window=129, n_keep_head=1, n_keep_tail=1)
+    idx = torch.full((2, 7), -1, dtype=torch.int32, device=DEV)
+    pooled = torch.zeros(2, 50, device=DEV)
+    R.retrieve_topk(bank.to(DEV), qs.to(DEV), 50, 7, idx, scale=0.5, pool_window=129, n_keep_head=1,
+                    n_keep_tail=1, pooled_score_out=pooled)
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    # every token has the same pooled score (the global maximum): ties go to the lowest indices
+    assert idx.cpu().tolist() == ref["idx"].tolist() == [[0, 1, 2, 3, 4, 5, 49]] * 2
+
+
 def test_retrieve_ties_take_lowest_index_and_k_ge_n():
     bank = torch.ones(1, 700, 32, dtype=torch.bfloat16)
     qs = torch.ones(1, 3, 32, dtype=torch.bfloat16)
