@@ -12,6 +12,14 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
 
+def pytest_sessionstart(session):
+    """Build the CUDA library and the CPU oracle if they are missing or older than their sources."""
+    from paper_2506_01215_b200 import build as rbuild
+    import oracle
+    rbuild.build()
+    oracle.build()
+
+
 def pytest_collection_modifyitems(config, items):
     import torch
 
