@@ -542,17 +542,7 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
     g_last_cuda_error = (int)cudaErrorInvalidValue;
     return REFORM_ERR_CUDA;
   }
-  int mode = 0;  // debugging aid: 1 = CUDA-core attention + tensor-core score pass, 2 = the reverse
-  if (const char* e = getenv("REFORM_SM100_MODE")) mode = atoi(e);
-  int rc = REFORM_OK;
-  if (!run_attention) {
-    // nothing to do here
-  } else if (mode == 1) {
-    reform_chunk_params q = *p;
-    q.flags |= REFORM_NO_SCORE;
-    rc = launch_chunk_simt(&q, lse, scale, st);
-    if (rc != REFORM_OK) return rc;
-  } else {
+  if (run_attention) {
     cudaFuncSetAttribute(attn2_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttn2SmemBytes);
     const int units = (p->Hq / p->Hkv) * ((p->Lc + kT - 1) / kT);
     dim3 grid((units + 1) / 2, p->B * p->Hkv);
@@ -560,21 +550,10 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
         tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
         p->dev_status);
     count_launch();
-    rc = check_launch();
+    int rc = check_launch();
     if (rc != REFORM_OK) return rc;
   }
   if (p->flags & REFORM_NO_SCORE) return REFORM_OK;
-  if (mode == 2) {
-    const float sl2 = scale_log2;
-    cudaFuncSetAttribute(score_simt_kernel<__nv_bfloat16, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)SimtSmem<128>::score_bytes);
-    dim3 grid2((n + kBN - 1) / kBN, p->B * p->Hkv);
-    score_simt_kernel<__nv_bfloat16, 128><<<grid2, kSimtThreads, SimtSmem<128>::score_bytes, st>>>(
-        (const __nv_bfloat16*)p->q, (const __nv_bfloat16*)p->k, lse, p->score, p->Hq, p->Hkv, p->Lc,
-        p->n_cache, p->cap, p->score_window, sl2, (p->flags & REFORM_SCORE_ACCUMULATE) ? 1 : 0);
-    count_launch();
-    return check_launch();
-  }
   cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScoreSmemBytes);
   dim3 grid2((n + kT - 1) / kT, p->B * p->Hkv);
   score_sm100_kernel<<<grid2, kSm100Threads, kScoreSmemBytes, st>>>(

@@ -326,7 +326,7 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
   if (!pooled) { pooled = reinterpret_cast<float*>(ws + off); off += retrieve_score_bytes(p); }
   rc = REFORM_ERR_UNSUPPORTED;
 #ifndef REFORM_NO_SM100
-  if (p->dtype == REFORM_BF16 && !getenv("REFORM_SCAN_NO_TCGEN05"))
+  if (p->dtype == REFORM_BF16)
     rc = launch_scan_sm100(p->bank, p->queries, ts, p->B, p->N, p->N_cap, p->E, p->nq, p->scale,
                            p->dev_status, st);
 #endif
