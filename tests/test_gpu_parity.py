@@ -45,6 +45,8 @@ CHUNK_CASES = [
     (2, 4, 4, 128, 257, 0, torch.bfloat16, 257),     # no GQA sharing, W = Lc
     (1, 4, 1, 128, 128, 512, torch.bfloat16, 64),    # cache much longer than chunk
     (1, 4, 2, 64, 96, 40, torch.bfloat16, 32),       # bf16 on the CUDA-core path (d = 64)
+    (3, 6, 2, 128, 300, 70, torch.bfloat16, 100),    # group of 3: tile pairs straddle heads, odd unit count
+    (1, 2, 2, 128, 1000, 0, torch.bfloat16, 128),    # pairs of consecutive query tiles with different walks
 ]
 
 
@@ -139,6 +141,27 @@ def test_alternative_compressors_through_the_same_calls():
     R.evict_topk(k.to(DEV), v.to(DEV), score, kd2, torch.zeros_like(kd2), torch.zeros(1, 2, 48, device=DEV),
                  500, 48, 16, 32, kept_idx=kept2)
     assert kept2.cpu()[0, 0].tolist() == list(range(16)) + list(range(468, 500))
+
+
+def test_chunk_step_extreme_logits():
+    """One key whose logit towers over everything seen before it (a jump of more than 100 in log2
+    units in the middle of the walk): the running maximum must be re-based without overflow, rows
+    that see the key return its value row, rows before it are untouched by it, nothing is NaN."""
+    q, k, v, carry = _case(1, 4, 2, 128, 400, 200, torch.bfloat16, seed=77)
+    q[..., 0] = 30.0
+    k[..., 0] = 0.0
+    j = 200 + 150                       # chunk row 150, in the second key tile of the chunk part
+    k[:, :, j, 0] = 30.0
+    out, lse, score = _run_chunk(q, k, v, carry, 200, 128, flags=0)
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all() and torch.isfinite(score[:, :, :600]).all()
+    o_ref, l_ref = oracle.attention(q, k, v, 200)
+    assert_outputs_close(out, o_ref, torch.bfloat16)
+    assert (lse.cpu().double() - l_ref).abs().max() < 2e-3
+    expect = v[:, :, j].double().repeat_interleave(2, dim=1)[:, :, None, :]
+    assert (out[:, :, 150:].cpu().double() - expect).abs().max() < 2e-2
+    s_ref = oracle.key_scores(q, k, 200, 128)
+    assert_scores_close(score[:, :, :600], s_ref[:, :, :600], 128 * 2 / 600)
+    assert abs(score[0, 0, j].item() - 256.0) < 0.3       # it takes all the mass of the 128 x 2 scoring rows
 
 
 def test_chunk_step_is_deterministic():
