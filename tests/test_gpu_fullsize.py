@@ -157,6 +157,84 @@ def test_retrieve_and_gather_full_size(name):
         assert torch.equal(dst[0][m].cpu().view(torch.int16), exp[0].view(torch.int16))
 
 
+def test_retrieval_bank_beyond_2_to_31_elements():
+    """Largest sizes: a ragged 2,500,037-row bank (2.56e9 elements, 5.1 GB) against the full oracle."""
+    w = dataclasses.replace(synth.WORKLOADS["retrieval_1m"], N=2_500_037, nq=2, k=4096, n_planted=32)
+    bank, qs, planted = synth.bank_and_queries(w, device=DEV)
+    assert bank.numel() > 2 ** 31
+    idx = torch.full((w.B, w.k), -1, dtype=torch.int32, device=DEV)
+    ts = torch.empty(w.B, w.N, device=DEV)
+    pooled = torch.empty(w.B, w.N, device=DEV)
+    p = dict(scale=w.sim_scale, pool_window=w.pool_window, n_keep_head=w.keep_head, n_keep_tail=w.keep_tail)
+    R.retrieve_topk(bank, qs, w.N, w.k, idx, token_score_out=ts, pooled_score_out=pooled, **p)
+    torch.cuda.synchronize()
+    assert R.device_error() == 0
+    ref = oracle.retrieve_topk(bank.cpu(), qs.cpu(), w.N, w.k, **p)
+    assert_scores_close(ts, ref["ts"], 1.0)
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    assert_index_sets_match(idx[0].cpu(), ref["idx"][0], ref["pooled"][0])
+    assert (ts[0].cpu()[torch.tensor(planted[0])] - w.rho).abs().max() < 5e-3
+
+
+def test_evict_32_layers_batched_bit_exact():
+    """Largest sizes: the batched call of config 3 (32 layers x 8 KV heads x 40,960 keys; K and V
+    of 2.7 GB each, byte offsets past 2^31) against the oracle's full sort."""
+    w = dataclasses.replace(synth.WORKLOADS["llama8b_128k"], B=32)
+    g = torch.Generator(device=DEV).manual_seed(5)
+    k = torch.randn(w.B, w.Hkv, w.cap, w.d, generator=g, device=DEV).to(w.dtype)
+    v = torch.randn(w.B, w.Hkv, w.cap, w.d, generator=g, device=DEV).to(w.dtype)
+    sc = torch.rand(w.B, w.Hkv, w.cap, generator=g, device=DEV)
+    kd = torch.zeros(w.B, w.Hkv, w.budget, w.d, dtype=w.dtype, device=DEV)
+    vd = torch.zeros_like(kd)
+    sd = torch.zeros(w.B, w.Hkv, w.budget, device=DEV)
+    kept = torch.zeros(w.B, w.Hkv, w.budget, dtype=torch.int32, device=DEV)
+    R.evict_topk(k, v, sc, kd, vd, sd, w.cap, w.budget, w.n_sink, w.n_recent, kept_idx=kept)
+    torch.cuda.synchronize()
+    assert R.device_error() == 0
+    ref = oracle.evict_topk(k.cpu(), v.cpu(), sc.cpu(), w.cap, w.budget, w.n_sink, w.n_recent,
+                            cap_dst=w.budget)
+    assert torch.equal(kept.cpu(), ref["kept_idx"])
+    assert torch.equal(kd.cpu().view(torch.int16), ref["k"].view(torch.int16))
+    assert torch.equal(vd.cpu().view(torch.int16), ref["v"].view(torch.int16))
+    assert torch.equal(sd.cpu().double(), ref["score"])
+
+
+def test_chunk_step_beyond_2_to_31_elements():
+    """Largest sizes: 5 sequences x 32 heads x 131,072 rows x 128 (2.7e9 elements of Q and of O) in
+    one call; sampled rows of the last sequence and head group, whose offsets pass 2^31."""
+    w = dataclasses.replace(synth.WORKLOADS["mistral7b_4x256k"], B=5, Lc=131072, budget=1024, T=262144)
+    G = w.Hq // w.Hkv
+    q, kc, vc = synth.chunk_qkv(w, 0, 1, device=DEV)
+    k0, v0, s0 = synth.cache_state(w, 0, device=DEV)
+    k = torch.cat([k0, kc], 2).contiguous()
+    v = torch.cat([v0, vc], 2).contiguous()
+    del kc, vc
+    assert q.numel() > 2 ** 31
+    carry = torch.cat([s0, torch.zeros(w.B, w.Hkv, w.Lc, device=DEV)], 2).contiguous()
+    score = carry.clone()
+    out = torch.empty_like(q)
+    lse = torch.empty(q.shape[:3], dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.chunk_step(q, k, v, out, score, w.budget, w.window, lse=lse, flags=R.SCORE_ACCUMULATE,
+                 dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    n = w.budget + w.Lc
+    new = score[:, :, :n].double().sum(-1) - carry[:, :, :w.budget].double().sum(-1)
+    assert torch.allclose(new, torch.full_like(new, float(w.window * G)), rtol=1e-3)
+    rows = [0, 1, 127, 128, 4095, 65535, 65536, 100000, w.Lc - 129, w.Lc - 2, w.Lc - 1]
+    for seq, g in ((4, 7), (0, 0)):
+        qs = q[seq:seq + 1, g * G:(g + 1) * G].cpu().contiguous()
+        ks = k[seq:seq + 1, g:g + 1].cpu().contiguous()
+        vs = v[seq:seq + 1, g:g + 1].cpu().contiguous()
+        o_ref, l_ref = oracle.attention(qs, ks, vs, w.budget, rows=rows)
+        assert_outputs_close(out[seq:seq + 1, g * G:(g + 1) * G][:, :, rows], o_ref, w.dtype)
+        assert (lse[seq:seq + 1, g * G:(g + 1) * G][:, :, rows].cpu().double() - l_ref).abs().max() < 2e-3
+        s_ref = oracle.key_scores(qs, ks, w.budget, w.window, score_in=carry[seq:seq + 1, g:g + 1].cpu(),
+                                  accumulate=True)
+        assert_scores_close(score[seq:seq + 1, g:g + 1, :n], s_ref[:, :, :n], w.window * G / n)
+
+
 def test_recurrent_pipeline_full_size_keeps_needles():
     """Config 2 end to end on the GPU (4 chunk steps + evictions): positions are carried through the
     compaction, every needle is still in every KV head's cache at the end, mass is conserved."""
