@@ -320,11 +320,14 @@ int reform_gather(const reform_gather_params* p, reform_stream_t stream);
  *   a' = a cos(angle) - b sin(angle);   b' = b cos(angle) + a sin(angle)
  * with pair i = (x[i], x[i + d/2]) (interleaved == 0, the rotate-half layout
  * of the Llama / Mistral family) or (x[2i], x[2i+1]) (interleaved != 0).
- * Angles are evaluated in fp64, the rotation in fp32, one rounding to dtype.
+ * Angles are reduced to [-pi, pi] in fp64 and their sine and cosine evaluated
+ * in fp32 (absolute error about 1e-7), the rotation in fp32, one rounding to
+ * dtype.
  *
  *   src [B,H,cap,d] in;  dst [B,H,cap,d] out (may be src: in place); rows
  *   outside the range are not touched.  theta_base 0 means 10000.
- * d * sizeof(dtype) must be a multiple of 32.
+ * d * sizeof(dtype) must be a multiple of 32 and d at most 512
+ * (REFORM_ERR_UNSUPPORTED otherwise).
  * ------------------------------------------------------------------------ */
 typedef struct reform_rope_params {
   size_t struct_size;

@@ -375,7 +375,7 @@ int reform_rope(const reform_rope_params* p, reform_stream_t stream) {
   if (p->B < 0 || p->H < 0 || p->d <= 0 || p->cap < 0 || p->row_begin < 0 || p->rows < 0 ||
       p->row_begin + p->rows > p->cap || p->pos_begin < 0 || !(p->theta_base >= 0.f))
     return REFORM_ERR_INVALID_ARG;
-  if ((p->d * elem_size(p->dtype)) % 32 != 0) return REFORM_ERR_UNSUPPORTED;
+  if ((p->d * elem_size(p->dtype)) % 32 != 0 || p->d / 2 > kRopeMaxPairs) return REFORM_ERR_UNSUPPORTED;
   if (!p->src || !p->dst || !aligned16(p->src) || !aligned16(p->dst)) return REFORM_ERR_INVALID_ARG;
   const double base = p->theta_base > 0.f ? (double)p->theta_base : 10000.0;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);

@@ -3,14 +3,22 @@
 // keeps un-rotated keys and row r of [cache ; chunk] is rotated by position
 // pos_begin + r when the step's operands are prepared).  HBM-bound: one read
 // and one write of the rotated rows.  The angle depends on (row, pair) only,
-// so a thread evaluates cos/sin once -- in fp64, positions reach 10^6 and an
-// fp32 angle would be off by 1e-2 rad there -- and reuses them for every
-// batch entry and head of that row.
+// so a thread evaluates cos/sin once and reuses them for every batch entry and
+// head of that row.  Positions reach 10^6, where an fp32 angle would be off by
+// 1e-2 rad, so the angle is reduced in fp64: the host passes each pair's
+// frequency in turns per position (fp64), the product with the position is
+// reduced to [-1/2, 1/2] turns in fp64, and only the reduced angle -- as an
+// fp32 value plus its fp32 remainder -- goes through the fp32 sincospi.
 #pragma once
 
 #include "common.cuh"
 
 namespace reform {
+
+constexpr int kRopeMaxPairs = 256;  // head dimensions up to 512
+struct RopeFreq {
+  double turns[kRopeMaxPairs];  // theta_base^(-2 i / d) / (2 pi)
+};
 
 // Thread = (row, group of NP consecutive pairs); block = 256 threads.
 //   half layout (interleaved == 0): pair i = (x[i], x[i + d/2]); a thread loads NP consecutive
@@ -19,7 +27,7 @@ namespace reform {
 template <typename T, bool INTERLEAVED>
 __global__ void __launch_bounds__(256)
 rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long long cap,
-            long long row_begin, long long rows, long long pos_begin, double log2_base) {
+            long long row_begin, long long rows, long long pos_begin, const __grid_constant__ RopeFreq freq) {
   constexpr int NP = 16 / (int)sizeof(T) / (INTERLEAVED ? 2 : 1);  // pairs per thread: one or two 16-byte vectors
   const int groups = (d / 2) / NP;                                  // thread groups per row
   const long long items = rows * groups;
@@ -31,10 +39,14 @@ rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long 
     float c[NP], s[NP];
 #pragma unroll
     for (int i = 0; i < NP; ++i) {
-      double sn, cs;
-      sincos(pos * exp2(-2.0 * (p0 + i) / d * log2_base), &sn, &cs);
-      c[i] = (float)cs;
-      s[i] = (float)sn;
+      const double t = pos * freq.turns[p0 + i];
+      const double fr = t - rint(t);           // [-1/2, 1/2] turns, exact
+      const float hi = (float)fr;
+      const float lo = (float)(fr - (double)hi) * 6.2831853071795865f;  // radians left over
+      float sn, cs;
+      sincospif(2.0f * hi, &sn, &cs);
+      c[i] = fmaf(-lo, sn, cs);                // first-order correction for the remainder
+      s[i] = fmaf(lo, cs, sn);
     }
 #pragma unroll 4
     for (int bh = 0; bh < BH; ++bh) {
@@ -77,11 +89,12 @@ inline int launch_rope(const void* src, void* dst, int BH, int d, long long cap,
   long long blocks = (items + 255) / 256;
   const long long cap_blocks = (long long)kNumSMs * 16;
   const int grid = (int)(blocks < cap_blocks ? blocks : cap_blocks);
-  const double log2_base = log2(base);
+  RopeFreq freq;
+  for (int i = 0; i < d / 2; ++i) freq.turns[i] = pow(base, -2.0 * i / d) / 6.283185307179586476925;
   if (interleaved)
-    rope_kernel<T, true><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, log2_base);
+    rope_kernel<T, true><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, freq);
   else
-    rope_kernel<T, false><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, log2_base);
+    rope_kernel<T, false><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, freq);
   count_launch();
   return check_launch();
 }

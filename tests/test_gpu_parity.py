@@ -494,7 +494,7 @@ def test_tiny_free_running_pipeline_with_driver():
 
 @pytest.mark.parametrize("dtype,d,interleaved,pos0", [
     (torch.bfloat16, 128, False, 0), (torch.bfloat16, 128, False, 1000000), (torch.bfloat16, 64, True, 40960),
-    (torch.float32, 64, False, 8191), (torch.float32, 32, True, 5),
+    (torch.float32, 64, False, 8191), (torch.float32, 32, True, 5), (torch.float32, 128, False, 1000000),
 ])
 def test_rope_matches_oracle(dtype, d, interleaved, pos0):
     g = torch.Generator().manual_seed(d + pos0 % 97)
