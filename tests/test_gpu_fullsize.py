@@ -235,10 +235,18 @@ def test_chunk_step_beyond_2_to_31_elements():
         assert_scores_close(score[seq:seq + 1, g:g + 1, :n], s_ref[:, :, :n], w.window * G / n)
 
 
-def test_recurrent_pipeline_full_size_keeps_needles():
-    """Config 2 end to end on the GPU (4 chunk steps + evictions): positions are carried through the
-    compaction, every needle is still in every KV head's cache at the end, mass is conserved."""
-    w = synth.WORKLOADS["llama8b_128k"]
+@pytest.mark.parametrize("name,accumulate,needles_must_survive", [
+    ("llama8b_128k", True, True), ("llama8b_1m_32l", False, True), ("llama8b_1m_32l", True, False)])
+def test_recurrent_pipeline_full_size_keeps_needles(name, accumulate, needles_must_survive):
+    """Configs 2 and 3 (one layer) end to end on the GPU: 4 and 32 chunk steps with their evictions.
+    Positions are carried through the compaction, mass is conserved, and every eviction equals the
+    oracle's full sort of the scores the GPU held before it (teacher forcing).  Every needle seen so
+    far is still in every KV head's cache after every step -- except in the 32-step run with
+    accumulated scores, where rows that have collected mass for many steps out-score a needle that
+    has been scored once (the oracle evicts it as well), so only the equality with the oracle is
+    asserted there."""
+    w = synth.WORKLOADS[name]
+    flags = R.SCORE_ACCUMULATE if accumulate else 0
     G = w.Hq // w.Hkv
     needles = set(synth.needle_positions(w))
     bufs = [[torch.zeros(w.B, w.Hkv, w.cap, w.d, dtype=w.dtype, device=DEV) for _ in range(2)] for _ in range(2)]
@@ -252,16 +260,24 @@ def test_recurrent_pipeline_full_size_keeps_needles():
         bufs[cur][1][:, :, n_cache:n_cache + w.Lc] = vc
         pos[cur][:, :, n_cache:n_cache + w.Lc] = torch.arange(step * w.Lc, (step + 1) * w.Lc, device=DEV,
                                                              dtype=torch.int32)
-        before = sc[cur][:, :, :n_cache].double().sum(-1)
-        R.chunk_step(q, bufs[cur][0], bufs[cur][1], out, sc[cur], n_cache, w.window, flags=R.SCORE_ACCUMULATE)
+        before = sc[cur][:, :, :n_cache].double().sum(-1) * (1 if accumulate else 0)
+        R.chunk_step(q, bufs[cur][0], bufs[cur][1], out, sc[cur], n_cache, w.window, flags=flags)
         after = sc[cur][:, :, :n_cache + w.Lc].double().sum(-1)
         assert torch.allclose(after - before, torch.full_like(after, float(w.window * G)), rtol=1e-3)
         nxt = 1 - cur
+        n_keys = n_cache + w.Lc
+        kept_idx = torch.zeros(w.B, w.Hkv, w.budget, dtype=torch.int32, device=DEV)
         n_cache = R.evict_topk(bufs[cur][0], bufs[cur][1], sc[cur], bufs[nxt][0], bufs[nxt][1], sc[nxt],
-                               n_cache + w.Lc, w.budget, w.n_sink, w.n_recent, pos_src=pos[cur], pos_dst=pos[nxt])
+                               n_keys, w.budget, w.n_sink, w.n_recent, pos_src=pos[cur], pos_dst=pos[nxt],
+                               kept_idx=kept_idx)
+        ref = oracle.evict_topk(torch.zeros(w.B, w.Hkv, n_keys, 8, dtype=w.dtype),
+                                torch.zeros(w.B, w.Hkv, n_keys, 8, dtype=w.dtype), sc[cur][:, :, :n_keys].cpu(),
+                                n_keys, w.budget, w.n_sink, w.n_recent, cap_dst=w.budget)
+        assert torch.equal(kept_idx.cpu()[:, :, :n_cache], ref["kept_idx"][:, :, :n_cache])
         cur = nxt
         kept = pos[cur][:, :, :n_cache].cpu()
         assert (kept[:, :, 1:] > kept[:, :, :-1]).all()               # order preserved
         seen = {p for p in needles if p < (step + 1) * w.Lc}
         for h in range(w.Hkv):
-            assert seen <= set(kept[0, h].tolist()), f"needle lost in head {h} at step {step}"
+            if needles_must_survive:
+                assert seen <= set(kept[0, h].tolist()), f"needle lost in head {h} at step {step}"
