@@ -46,12 +46,25 @@ __device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
 // S (or S^T) = A B^T for two K-major 128 x 128 bf16 tiles in shared memory: 8 MMAs of K = 16
 __device__ __forceinline__ void issue_kmajor_128x128x128(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
   constexpr uint32_t idesc = ptx::idesc_bf16(kT, kT, false, false);
+  const uint32_t a_lo = ptx::smem_desc_lo(a_smem, 16), b_lo = ptx::smem_desc_lo(b_smem, 16);
+  ptx::mma_ss_c<0>(d_tmem, a_lo, b_lo, ptx::kDescHiSw128, idesc);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;  // 64-column box, then 32 B per K = 16 step
-    ptx::mma_ss(d_tmem, ptx::smem_desc_sw128(a_smem + off, 16, 1024),
-                ptx::smem_desc_sw128(b_smem + off, 16, 1024), idesc, k > 0);
+  for (int k = 1; k < 8; ++k) {
+    constexpr uint32_t box = kHalfBytes >> 4;              // 64-column box, then 32 B per K = 16 step
+    const uint32_t off = (k >> 2) * box + (k & 3) * 2;
+    ptx::mma_ss_c<1>(d_tmem, a_lo + off, b_lo + off, ptx::kDescHiSw128, idesc);
   }
+}
+
+// O (+)= P V for keys [16 * K0, 16 * K0 + 64) of a key tile: P (bf16) from TMEM, V MN-major in shared memory
+template <int K0>
+__device__ __forceinline__ void issue_pv_half(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_lo, bool first) {
+  constexpr uint32_t idesc = ptx::idesc_bf16(kT, kT, false, true);
+  if (K0 == 0 && first) ptx::mma_ts_c<0>(o_tmem, p_tmem, v_lo, ptx::kDescHiSw128, idesc);
+  else ptx::mma_ts_c<1>(o_tmem, p_tmem + 8 * K0, v_lo + K0 * 128, ptx::kDescHiSw128, idesc);
+#pragma unroll
+  for (int k = K0 + 1; k < K0 + 4; ++k)
+    ptx::mma_ts_c<1>(o_tmem, p_tmem + 8 * k, v_lo + k * 128, ptx::kDescHiSw128, idesc);
 }
 
 // ---------------------------------------------------------------------------
@@ -186,7 +199,6 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
       }
     } else if (warp == 9 && lane == 0) {
-      constexpr uint32_t idesc_pv = ptx::idesc_bf16(kT, kT, false, true);  // V is MN-major
       const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK), aV = ptx::smem_u32(sV);
       const uint32_t tS0 = tmem_base, tO0 = tmem_base + 128, tS1 = tmem_base + 256, tO1 = tmem_base + 384;
       bool ok = ptx::mbar_wait(q_full, 0, abort_flag) && ptx::mbar_wait(k_full, 0, abort_flag);
@@ -207,16 +219,11 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!ptx::mbar_wait(p_ready + 0, j & 1, abort_flag)) break;
         if (!ptx::mbar_wait(v_full + s, ph, abort_flag)) break;
         ptx::tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          ptx::mma_ts(tO0, tS0 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
-                      idesc_pv, (j > 0) || (k > 0));
+        const uint32_t v_lo = ptx::smem_desc_lo(aV + s * kTileBytes, kHalfBytes);
+        issue_pv_half<0>(tO0, tS0, v_lo, j == 0);
         if (!ptx::mbar_wait(p_ready + 1, j & 1, abort_flag)) break;
         ptx::tc_fence_after();
-#pragma unroll
-        for (int k = 4; k < 8; ++k)
-          ptx::mma_ts(tO0, tS0 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
-                      idesc_pv, 1);
+        issue_pv_half<4>(tO0, tS0, v_lo, false);
         if (j + 1 < n_kt0) {
           if (!ptx::mbar_wait(k_full + s1, ph1, abort_flag)) break;
           ptx::tc_fence_after();
@@ -229,16 +236,10 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (j < n_kt1) {
           if (!ptx::mbar_wait(p_ready + 2, j & 1, abort_flag)) break;
           ptx::tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            ptx::mma_ts(tO1, tS1 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
-                        idesc_pv, (j > 0) || (k > 0));
+          issue_pv_half<0>(tO1, tS1, v_lo, j == 0);
           if (!ptx::mbar_wait(p_ready + 3, j & 1, abort_flag)) break;
           ptx::tc_fence_after();
-#pragma unroll
-          for (int k = 4; k < 8; ++k)
-            ptx::mma_ts(tO1, tS1 + 8 * k, ptx::smem_desc_sw128(aV + s * kTileBytes + k * 2048, kHalfBytes, 1024),
-                        idesc_pv, 1);
+          issue_pv_half<4>(tO1, tS1, v_lo, false);
         }
         ptx::mma_commit(v_empty + s);
         if (j + 1 < n_kt1) {
