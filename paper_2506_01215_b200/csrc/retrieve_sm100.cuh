@@ -84,14 +84,14 @@ scan_sm100_kernel(const __grid_constant__ CUtensorMap tmBank, const __grid_const
       ptx::prefetch_tmap(&tmQ);
       ptx::mbar_expect_tx(q_full, (uint32_t)KB * q_box_bytes);
       for (int kb = 0; kb < KB; ++kb) ptx::tma_load_3d(sQ + (size_t)kb * q_box_bytes, &tmQ, q_full, 64 * kb, 0, b);
-      uint32_t it = 0;  // stage uses so far
+      uint32_t it = 0, s = 0, ph = 0;  // stage uses so far; stage and phase of the next one
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < tiles_per_seq; tile += gridDim.x) {
         for (int kb = 0; kb < KB; ++kb, ++it) {
-          const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
           if (!ptx::mbar_wait(a_empty + s, ph ^ 1, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(a_full + s, kScanStageBytes);
           ptx::tma_load_3d(sA + (size_t)s * kScanStageBytes, &tmBank, a_full + s, 64 * kb, tile * kScanTileTokens, b);
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1; }
         }
       }
       if (*abort_flag) {  // let copies in flight land before shared memory is released
@@ -108,19 +108,27 @@ scan_sm100_kernel(const __grid_constant__ CUtensorMap tmBank, const __grid_const
       const uint32_t idesc = ptx::idesc_bf16(128, n_pad, false, false);
       const uint32_t aQ = ptx::smem_u32(sQ), aA = ptx::smem_u32(sA);
       bool ok = ptx::mbar_wait(q_full, 0, abort_flag);
-      uint32_t it = 0, i = 0;
+      // the tensor pipe runs only while this thread issues: stage, phase and descriptor words are
+      // stepped, not recomputed, and the accumulate flag of all but a tile's first MMA is a constant
+      const uint32_t a_lo0 = ptx::smem_desc_lo(aA, 16), q_lo0 = ptx::smem_desc_lo(aQ, 16);
+      const uint32_t stage_step = kScanStageBytes >> 4, q_step = (uint32_t)q_box_bytes >> 4;
+      uint32_t i = 0, s = 0, ph = 0, a_lo = a_lo0;
       for (int tile = blockIdx.x; ok && tile < tiles_per_seq; tile += gridDim.x, ++i) {
         const uint32_t buf = i & 1;
+        const uint32_t d = tmem_base + buf * 64;
         if (!ptx::mbar_wait(acc_empty + buf, ((i >> 1) & 1) ^ 1, abort_flag)) break;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
-          const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
+        uint32_t q_lo = q_lo0;
+        for (int kb = 0; kb < KB; ++kb) {
           if (!ptx::mbar_wait(a_full + s, ph, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after();
+          if (kb == 0) ptx::mma_ss_c<0>(d, a_lo, q_lo, ptx::kDescHiSw128, idesc);
+          else ptx::mma_ss_c<1>(d, a_lo, q_lo, ptx::kDescHiSw128, idesc);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            ptx::mma_ss(tmem_base + buf * 64, ptx::smem_desc_sw128(aA + s * kScanStageBytes + k * 32, 16, 1024),
-                        ptx::smem_desc_sw128(aQ + kb * q_box_bytes + k * 32, 16, 1024), idesc, (kb > 0) || (k > 0));
+          for (int k = 1; k < 4; ++k) ptx::mma_ss_c<1>(d, a_lo + 2 * k, q_lo + 2 * k, ptx::kDescHiSw128, idesc);
           ptx::mma_commit(a_empty + s);
+          q_lo += q_step;
+          a_lo += stage_step;
+          if (++s == (uint32_t)n_stages) { s = 0; ph ^= 1; a_lo = a_lo0; }
         }
         if (ok) ptx::mma_commit(acc_full + buf);
       }
