@@ -213,11 +213,11 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ptx::mma_commit(k_empty + 0);
       }
       for (int j = 0; ok && j < n_kt0; ++j) {
-        const int s = j & 1, ph = (j >> 1) & 1;
-        const int s1 = (j + 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+        const int s = j & 1, s1 = (j + 1) & 1;
         // tile 0: O0 += P0 V[j], then S0 = Q0 K[j+1]^T
+        // (thread 0 of tile 0's warpgroup has seen V[j] before its first arrival on p_ready and
+        // K[j+1] before its second: a wait costs this thread one to two MMAs even when satisfied)
         if (!ptx::mbar_wait(p_ready + 0, j & 1, abort_flag)) break;
-        if (!ptx::mbar_wait(v_full + s, ph, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t v_lo = ptx::smem_desc_lo(aV + s * kTileBytes, kHalfBytes);
         issue_pv_half<0>(tO0, tS0, v_lo, j == 0);
@@ -225,8 +225,6 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ptx::tc_fence_after();
         issue_pv_half<4>(tO0, tS0, v_lo, false);
         if (j + 1 < n_kt0) {
-          if (!ptx::mbar_wait(k_full + s1, ph1, abort_flag)) break;
-          ptx::tc_fence_after();
           issue_kmajor_128x128x128(tS0, aQ, aK + s1 * kTileBytes);
           ptx::mma_commit(s_full + 0);
         } else {
@@ -328,8 +326,15 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ptx::tmem_st32(tS + 32 * half, pk);
         ptx::tmem_st_wait();
         ptx::tc_fence_before();
+        if (threadIdx.x == 0) {  // on behalf of the MMA issuer: the operands its next MMAs read are in shared memory
+          const int jn = j + 1;
+          const bool there = half == 0 ? ptx::mbar_wait(v_full + (j & 1), (j >> 1) & 1, abort_flag)
+                                       : (jn >= tile.n_kt || ptx::mbar_wait(k_full + (jn & 1), (jn >> 1) & 1, abort_flag));
+          if (!there) { ok = false; break; }
+        }
         ptx::mbar_arrive(p_ready + 2 * t + half);
       }
+      if (!ok) break;
     }
     if (ok && ptx::mbar_wait(o_full + t, 0, abort_flag)) {
       ptx::tc_fence_after();
