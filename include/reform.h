@@ -293,6 +293,11 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
  * row_bytes is a multiple of 16.  An index outside [0, n_rows) zero-fills its
  * row and sets REFORM_DEV_BAD_INDEX in *dev_status; no out-of-range access
  * is made.
+ * src is any address the device can read: device memory, or page-locked host
+ * memory under unified addressing (cudaHostAlloc, cudaHostRegister).  In the
+ * second case only the k selected rows of each sequence cross the bus, which
+ * is what a caller wants whose input embeddings of a million-token context
+ * stay in host memory.  idx and dst are device memory.
  * ------------------------------------------------------------------------ */
 typedef struct reform_gather_params {
   size_t struct_size;

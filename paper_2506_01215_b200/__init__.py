@@ -155,11 +155,12 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"reform kernels take float32 or bfloat16 tensors, got {t.dtype}")
 
 
-def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+def _ptr(t: Optional[torch.Tensor], pinned_ok: bool = False) -> Optional[int]:
     if t is None:
         return None
-    if not t.is_cuda:
-        raise ValueError("reform entry points take device tensors")
+    if not t.is_cuda and not (pinned_ok and t.is_pinned()):
+        raise ValueError("reform entry points take device tensors" +
+                         (" (or, here, page-locked host memory)" if pinned_ok else ""))
     if not t.is_contiguous():
         raise ValueError("reform entry points take contiguous tensors")
     return t.data_ptr()
@@ -280,11 +281,12 @@ def retrieve_topk(bank, queries, N: int, k: int, idx_out, *, scale: float = 1.0,
 
 
 def gather(src, idx, dst, *, dev_status=None, stream=None):
-    """reform_gather: src [B,n_rows,D], idx [B,k] int32, dst [B,k,D]."""
+    """reform_gather: src [B,n_rows,D] (device, or pinned host memory read in place), idx [B,k]
+    int32, dst [B,k,D]."""
     B, n_rows, D = src.shape
     k = idx.shape[1]
-    p = GatherParams(ctypes.sizeof(GatherParams), B, k, n_rows, D * src.element_size(), _ptr(src),
-                     _ptr(idx), _ptr(dst), _ptr(dev_status))
+    p = GatherParams(ctypes.sizeof(GatherParams), B, k, n_rows, D * src.element_size(),
+                     _ptr(src, pinned_ok=True), _ptr(idx), _ptr(dst), _ptr(dev_status))
     _check("reform_gather", lib().reform_gather(ctypes.byref(p), _stream(stream)))
 
 

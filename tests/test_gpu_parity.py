@@ -490,6 +490,19 @@ def test_tiny_free_running_pipeline_with_driver():
     assert_scores_close(cache.score[cache.cur][:, :, :n_cache], cs[:, :, :n_cache], 1e-3) if same == 1.0 else None
 
 
+def test_gather_reads_rows_out_of_pinned_host_memory():
+    """The gather source may stay in page-locked host memory: same bytes as from device memory."""
+    g = torch.Generator().manual_seed(11)
+    src = torch.randn(2, 5000, 1024, generator=g).to(torch.bfloat16).pin_memory()
+    idx = torch.stack([torch.sort(torch.randperm(5000, generator=g)[:300]).values for _ in range(2)]).to(torch.int32)
+    dst = torch.zeros(2, 300, 1024, dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.gather(src, idx.to(DEV), dst, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(dst.cpu().view(torch.int16), oracle.gather(src, idx).view(torch.int16))
+
+
 # ------------------------------------------------------------------- rope
 
 @pytest.mark.parametrize("dtype,d,interleaved,pos0", [
