@@ -490,6 +490,44 @@ def test_tiny_free_running_pipeline_with_driver():
     assert_scores_close(cache.score[cache.cur][:, :, :n_cache], cs[:, :, :n_cache], 1e-3) if same == 1.0 else None
 
 
+def test_chunk_step_seeded_random_shapes():
+    """Sixty seeded shapes of the tensor-core chunk step (group sizes 1-8, chunk lengths and cache
+    sizes on and off the 128 tile grid, windows 1 .. Lc, padded capacity, both score modes), each
+    compared with the oracle in full."""
+    import random
+    rnd = random.Random(20250601)
+    for case in range(60):
+        B = rnd.choice([1, 1, 2]); Hkv = rnd.choice([1, 2, 3]); G = rnd.choice([1, 2, 3, 4, 5, 8])
+        Lc = rnd.choice([1, 2, 5, 17, 64, 127, 128, 129, 200, 256, 257, 300, 383, 384, 500, 641])
+        n_cache = rnd.choice([0, 0, 1, 63, 128, 130, 255, 256, 300, 512, 777])
+        if Lc * G <= 16:
+            Lc += 17                                   # decode-shaped steps have tests of their own
+        W = rnd.choice([1, min(Lc, 7), min(Lc, 128), Lc])
+        cap = n_cache + Lc + rnd.choice([0, 5, 64])
+        acc = rnd.choice([True, False])
+        g = torch.Generator().manual_seed(case * 7919 + 13)
+        q = (torch.randn(B, Hkv * G, Lc, 128, generator=g) * rnd.choice([1.0, 1.0, 3.0])).to(torch.bfloat16)
+        k = torch.randn(B, Hkv, cap, 128, generator=g).to(torch.bfloat16)
+        v = torch.randn(B, Hkv, cap, 128, generator=g).to(torch.bfloat16)
+        carry = torch.rand(B, Hkv, cap, generator=g)
+        qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+        score = carry.clone().to(DEV)
+        out = torch.empty_like(qd)
+        lse = torch.empty(B, Hkv * G, Lc, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        R.chunk_step(qd, kd, vd, out, score, n_cache, W, lse=lse,
+                     flags=R.SCORE_ACCUMULATE if acc else 0, dev_status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        n = n_cache + Lc
+        o_ref, l_ref = oracle.attention(q, k[:, :, :n].contiguous(), v[:, :, :n].contiguous(), n_cache)
+        assert_outputs_close(out, o_ref, torch.bfloat16)
+        assert (lse.cpu().double() - l_ref).abs().max() < 3e-3, case
+        s_ref = oracle.key_scores(q, k[:, :, :n].contiguous(), n_cache, W,
+                                  score_in=carry[:, :, :n].contiguous(), accumulate=acc)
+        assert_scores_close(score[:, :, :n], s_ref[:, :, :n], W * G / n)
+
+
 def test_gather_reads_rows_out_of_pinned_host_memory():
     """The gather source may stay in page-locked host memory: same bytes as from device memory."""
     g = torch.Generator().manual_seed(11)
