@@ -18,9 +18,11 @@
  *
  * Conventions common to every call
  *   - All tensor pointers are DEVICE pointers unless a field says "host".
- *     The caller owns every buffer; the library allocates nothing, keeps no
- *     pointer after the call returns and holds no global state besides a
- *     per-thread record of the last CUDA error and a launch counter.
+ *     The caller owns every buffer; the library allocates nothing and keeps
+ *     no pointer after the call returns.  Its global state is: a per-thread
+ *     record of the last CUDA error, a launch counter, one error word per
+ *     device (reform_device_error) and, per device, the fixed scratch array
+ *     of reform_evict_topk_static (REFORM_EVICT_STATIC_BYTES).
  *   - Work is enqueued on the caller's stream and the call returns without
  *     synchronising.  Results are valid once the stream reaches that point.
  *   - Tensors are dense, row-major, innermost dimension contiguous; device
@@ -36,7 +38,11 @@
  *     bytes, 256-byte aligned, private to the call while it is in flight.
  *   - Return value: REFORM_OK or a negative REFORM_ERR_* code.  On any error
  *     nothing has been launched.
- *   - Indices are int32.  NaN inputs are outside the contract.
+ *   - Indices are int32.  NaN inputs are outside the contract.  Batched
+ *     calls take at most 65,535 (sequence, head) pairs: B * Hq for the chunk
+ *     step, B * Hkv for the eviction, B for the retrieval; more is
+ *     REFORM_ERR_INVALID_ARG.  A workspace-size query returns 0 for arguments
+ *     the call itself would reject.
  */
 #ifndef REFORM_H_
 #define REFORM_H_
@@ -126,8 +132,8 @@ size_t reform_chunk_step_workspace_size(const reform_chunk_params* p);
 int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------
- * reform_evict_topk -- Sec. 3.1 cache compression (Fig. 1 step 3), "always
- * keep the initial and recent tokens" (Sec. 4 "Common setup").
+ * reform_evict_topk -- Sec. 3.1 cache compression (Fig. 1 step 3); the initial
+ * and the most recent rows are never evicted (Sec. 4, common setup).
  *
  * Independently for every (b, KV head): if n_keys <= budget all rows are
  * kept.  Otherwise the first n_sink and last n_recent rows are kept, plus the
@@ -208,8 +214,10 @@ int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t strea
  *
  * For every b, chunk token t and selected (kind, head, slot):
  *   bank[b, token_offset + t, slot*d : (slot+1)*d] = x / max(||x||_2, eps)
- * with x the d-vector of that head's Q, K or V state for token t; norms in
- * fp32, one rounding (nearest-even) to the bank dtype.
+ * with x the d-vector of that head's Q, K or V state for token t.  Norm and
+ * quotient are computed in fp32 for a bf16 bank and in fp64 for an fp32 bank,
+ * then rounded once (nearest-even) to the bank dtype: every element is within
+ * one unit in the last place of the exact quotient.
  *
  *   q_state [B,Hq,Lc,d]; k_state, v_state [B,Hkv,Lc,d]  in; a kind that no
  *                         selection uses may be NULL
@@ -285,8 +293,8 @@ size_t reform_retrieve_topk_workspace_size(const reform_retrieve_params* p);
 int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------
- * reform_gather -- Sec. 3.3 "gather the corresponding input embeddings"
- * (Alg. 1, GatherRelevant).
+ * reform_gather -- Sec. 3.3, collecting the input embeddings of the selected
+ * tokens (Alg. 1, GatherRelevant).
  *
  *   dst[b, r, :] = src[b, idx[b, r], :]      r in [0, k)
  *   src [B,n_rows,row_bytes] in; idx [B,k] int32 in; dst [B,k,row_bytes] out
@@ -314,8 +322,8 @@ typedef struct reform_gather_params {
 int reform_gather(const reform_gather_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------
- * reform_rope -- Sec. 3.1: "after compression, we reassign the position IDs so
- * that the tokens in the compressed cache have consecutive position IDs".
+ * reform_rope -- Sec. 3.1, position re-assignment after compression: the rows
+ * that survive an eviction are renumbered 0, 1, 2, ... in cache order.
  * The cache therefore keeps un-rotated keys, and a step rotates its operands
  * with the ids of the moment: cache row r at position r, chunk row i at
  * n_cache + i (queries likewise).  This call applies the rotary embedding to

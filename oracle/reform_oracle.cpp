@@ -12,9 +12,9 @@
 // Operations (section / algorithm of the paper each one follows):
 //   oracle_attention      Sec. 3.1 + Fig. 1 step (1): a chunk's queries attend
 //                         causally over [compressed cache ; chunk].
-//   oracle_key_scores     Sec. 3.1 "attention-based token eviction following
-//                         H2O"; Sec. 4 common setup (scores from the last 128
-//                         queries of a chunk): attention mass per key.
+//   oracle_key_scores     Sec. 3.1 (eviction by attention mass, the H2O
+//                         criterion); Sec. 4 common setup (scores from the last
+//                         128 queries of a chunk): attention mass per key.
 //   oracle_evict_topk     Sec. 3.1 / Fig. 1 step (3): keep heavy hitters plus
 //                         the initial and recent tokens; order preserved so
 //                         position ids can be re-assigned consecutively.
@@ -24,14 +24,14 @@
 //                         cosine scan, max over query tokens, max-pool over
 //                         adjacent tokens, top-k with first/last tokens kept.
 //   oracle_gather         Sec. 3.3 / Alg. 1 GatherRelevant: row gather.
-//   oracle_rope           Sec. 3.1 "reassign the position IDs ... consecutive": rotary
+//   oracle_rope           Sec. 3.1, position re-assignment after compression: rotary
 //                         embedding at consecutive positions.
 //
 // Readings of the paper that it does not fix (reduction over the GQA group is
 // a sum, carried scores add, ties go to the lowest index, forced tokens count
 // toward the budget) are parameters or documented where they apply.
 // "parity unpinned" by the paper itself: the choice of sum over the GQA group
-// and of accumulation across chunks (the paper only says "following H2O").
+// and of accumulation across chunks (the paper only names the H2O criterion).
 
 #include <algorithm>
 #include <atomic>

@@ -9,7 +9,20 @@
 
 namespace reform {
 
-constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multiples of this
+// Streaming multiprocessors of the current device (148 on a B200: 2 dies x 74); grids are sized in
+// multiples of this.  Queried once per device and cached.
+inline int num_sms() {
+  constexpr int kMaxDevices = 64;
+  static int cache[kMaxDevices] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  int n = cache[dev];
+  if (n <= 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cache[dev] = n;
+  }
+  return n;
+}
 
 // Per-thread record of the last failing CUDA call and a process-wide launch counter.
 extern thread_local int g_last_cuda_error;

@@ -51,10 +51,22 @@ struct Vec4<__nv_bfloat16> {
   }
 };
 
+// Arithmetic type of the norm and the quotient.  A bf16 bank takes fp32 (its 8-bit significand
+// hides fp32 rounding: the result is within one bf16 unit of the exact quotient).  An fp32 bank
+// takes fp64, so that the single rounding to fp32 is the only error (within one fp32 unit).
+template <typename T>
+struct EmbedAcc { using type = float; };
+template <>
+struct EmbedAcc<float> { using type = double; };
+
+__device__ __forceinline__ float embed_norm(float ss, float eps) { return fmaxf(sqrtf(ss), eps); }
+__device__ __forceinline__ double embed_norm(double ss, float eps) { return fmax(sqrt(ss), (double)eps); }
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 embed_append_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, int E,
                     long long N_cap, long long token_offset, float eps) {
+  using Acc = typename EmbedAcc<T>::type;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -68,23 +80,26 @@ embed_append_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, in
     const T* x = reinterpret_cast<const T*>(sel.src[s]) +
                  (((long long)b * sel.H[s] + sel.head[s]) * Lc + t) * d;
     float v[kEmbedMaxVec][4];
-    float ss = 0.f;
+    Acc ss = 0;
 #pragma unroll
     for (int c = 0; c < kEmbedMaxVec; ++c) {
       int vi = lane + 32 * c;
       if (vi < nvec) {
         Vec4<T>::load(x + 4 * vi, v[c]);
-        ss += v[c][0] * v[c][0] + v[c][1] * v[c][1] + v[c][2] * v[c][2] + v[c][3] * v[c][3];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ss += (Acc)v[c][i] * (Acc)v[c][i];
       }
     }
-    ss = warp_sum(ss);
-    float nrm = fmaxf(sqrtf(ss), eps);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    const Acc nrm = embed_norm(ss, eps);
     T* y = bank + ((long long)b * N_cap + token_offset + t) * E + (long long)sel.slot[s] * d;
 #pragma unroll
     for (int c = 0; c < kEmbedMaxVec; ++c) {
       int vi = lane + 32 * c;
       if (vi < nvec) {
-        float o[4] = {v[c][0] / nrm, v[c][1] / nrm, v[c][2] / nrm, v[c][3] / nrm};
+        float o[4] = {(float)((Acc)v[c][0] / nrm), (float)((Acc)v[c][1] / nrm), (float)((Acc)v[c][2] / nrm),
+                      (float)((Acc)v[c][3] / nrm)};
         Vec4<T>::store(y + 4 * vi, o);
       }
     }
@@ -99,6 +114,7 @@ template <typename T, int LP>
 __global__ void __launch_bounds__(256)
 embed_append_vec_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d, int E,
                         long long N_cap, long long token_offset, float eps) {
+  using Acc = typename EmbedAcc<T>::type;
   constexpr int VPW = 32 / LP, U = 4, EPC = 16 / (int)sizeof(T);
   const int lane = threadIdx.x & 31;
   const int sub = lane % LP, which = lane / LP;
@@ -129,19 +145,25 @@ embed_append_vec_kernel(EmbedSel sel, T* __restrict__ bank, int B, int Lc, int d
     for (int u = 0; u < U; ++u) {
       float f[EPC];
       const T* e = reinterpret_cast<const T*>(&x[u]);
-      float ss = 0.f;
+      Acc ss = 0;
 #pragma unroll
       for (int i = 0; i < EPC; ++i) {
         f[i] = to_float(e[i]);
-        ss = fmaf(f[i], f[i], ss);
+        ss += (Acc)f[i] * (Acc)f[i];
       }
 #pragma unroll
       for (int o = LP / 2; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      const float inv = 1.0f / fmaxf(sqrtf(ss), eps);
       uint4 w;
       T* o4 = reinterpret_cast<T*>(&w);
+      if (sizeof(T) == 4) {  // fp32 bank: fp64 quotient, one rounding
+        const Acc nrm = embed_norm(ss, eps);
 #pragma unroll
-      for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>(f[i] * inv);
+        for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>((float)((Acc)f[i] / nrm));
+      } else {
+        const float inv = 1.0f / embed_norm((float)ss, eps);
+#pragma unroll
+        for (int i = 0; i < EPC; ++i) o4[i] = from_float<T>(f[i] * inv);
+      }
       if (ok[u]) __stcs(reinterpret_cast<uint4*>(y[u]), w);
     }
   }
@@ -158,7 +180,7 @@ inline int launch_embed(const EmbedSel& sel, void* bank, int B, int Lc, int d, i
   if (vec_ok) {
     long long per_warp = (32 / chunks) * 4;
     long long blocks = (items + 8 * per_warp - 1) / (8 * per_warp);
-    long long cap = (long long)kNumSMs * 8;
+    long long cap = (long long)num_sms() * 8;
     int grid = (int)(blocks < cap ? blocks : cap);
 #define REFORM_EMBED_CASE(LP)                                                                          \
   case LP:                                                                                             \
@@ -176,7 +198,7 @@ inline int launch_embed(const EmbedSel& sel, void* bank, int B, int Lc, int d, i
     return check_launch();
   }
   long long blocks = (items + 7) / 8;  // 8 warps per block
-  long long cap = (long long)kNumSMs * 16;
+  long long cap = (long long)num_sms() * 16;
   int grid = (int)(blocks < cap ? blocks : cap);
   embed_append_kernel<T><<<grid, 256, 0, st>>>(sel, (T*)bank, B, Lc, d, E, N_cap, token_offset, eps);
   count_launch();

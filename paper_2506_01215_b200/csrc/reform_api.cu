@@ -52,12 +52,23 @@ static bool chunk_uses_sm100(const reform_chunk_params* p) {
 #endif
 }
 
-static int validate_chunk(const reform_chunk_params* p) {
+// (batch, head) pairs index gridDim.y of the chunk-step kernels
+constexpr long long kMaxGridY = 65535;
+
+// Shape checks shared by the workspace-size query and the launch.
+static int validate_chunk_shape(const reform_chunk_params* p) {
   if (!p || p->struct_size != sizeof(reform_chunk_params)) return REFORM_ERR_INVALID_ARG;
   if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
   if (p->B < 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv != 0) return REFORM_ERR_INVALID_ARG;
+  if ((long long)p->B * p->Hq > kMaxGridY) return REFORM_ERR_INVALID_ARG;
   if (p->Lc < 0 || p->n_cache < 0 || (long long)p->n_cache + p->Lc > p->cap) return REFORM_ERR_INVALID_ARG;
   if (p->d != 64 && p->d != 128) return REFORM_ERR_UNSUPPORTED;
+  return REFORM_OK;
+}
+
+static int validate_chunk(const reform_chunk_params* p) {
+  int rc = validate_chunk_shape(p);
+  if (rc != REFORM_OK) return rc;
   if (!(p->flags & REFORM_NO_SCORE)) {
     if (p->Lc > 0 && (p->score_window < 1 || p->score_window > p->Lc)) return REFORM_ERR_INVALID_ARG;
     if (!p->score) return REFORM_ERR_INVALID_ARG;
@@ -86,8 +97,8 @@ using namespace reform;
 extern "C" {
 
 size_t reform_chunk_step_workspace_size(const reform_chunk_params* p) {
-  if (!p || p->struct_size != sizeof(reform_chunk_params)) return 0;
-  if (p->B <= 0 || p->Hq <= 0 || p->Lc <= 0) return 0;
+  if (validate_chunk_shape(p) != REFORM_OK) return 0;
+  if (p->B == 0 || p->Lc == 0) return 0;
   return chunk_workspace_bytes(p);
 }
 
@@ -123,6 +134,7 @@ static int validate_evict(const reform_evict_params* p) {
   if (!p || p->struct_size != sizeof(reform_evict_params)) return REFORM_ERR_INVALID_ARG;
   if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
   if (p->B < 0 || p->Hkv <= 0 || p->d <= 0) return REFORM_ERR_INVALID_ARG;
+  if ((long long)p->B * p->Hkv > kMaxGridY) return REFORM_ERR_INVALID_ARG;
   if (((size_t)p->d * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
   if (p->n_keys < 0 || p->n_keys > p->cap_src || p->budget < 0) return REFORM_ERR_INVALID_ARG;
   if (p->n_sink < 0 || p->n_recent < 0 || (long long)p->n_sink + p->n_recent > p->budget)
@@ -281,7 +293,8 @@ int reform_embed_append(const reform_embed_params* p, reform_stream_t stream) {
 static int validate_retrieve(const reform_retrieve_params* p) {
   if (!p || p->struct_size != sizeof(reform_retrieve_params)) return REFORM_ERR_INVALID_ARG;
   if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
-  if (p->B < 0 || p->N < 0 || p->N > p->N_cap || p->N > 0x7fffffffLL || p->E <= 0 || p->nq < 1)
+  if (p->B < 0 || p->B > kMaxGridY || p->N < 0 || p->N > p->N_cap || p->N > 0x7fffffffLL || p->E <= 0 ||
+      p->nq < 1)
     return REFORM_ERR_INVALID_ARG;
   if ((p->E * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
   if (p->pool_window < 1 || p->pool_window % 2 == 0) return REFORM_ERR_INVALID_ARG;

@@ -145,7 +145,7 @@ inline void launch_scan_mma_nt(const void* bank, const void* queries, float* ts,
   size_t smem = (size_t)8 * NT * E * 2;
   cudaFuncSetAttribute(scan_mma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   long long blocks = (tiles + 7) / 8;
-  long long cap = (long long)kNumSMs * (NT <= 2 ? 8 : (NT <= 4 ? 3 : 1));
+  long long cap = (long long)num_sms() * (NT <= 2 ? 8 : (NT <= 4 ? 3 : 1));
   dim3 grid((unsigned)(blocks < cap ? blocks : cap), B);
   scan_mma_kernel<NT><<<grid, 256, smem, st>>>((const __nv_bfloat16*)bank,
                                                (const __nv_bfloat16*)queries, ts, N, N_cap, E, nq,
@@ -163,7 +163,7 @@ inline int launch_scan(int dtype, const void* bank, const void* queries, float* 
     else launch_scan_mma_nt<8>(bank, queries, ts, B, N, N_cap, E, nq, scale, st);
   } else {
     long long blocks = ((long long)B * N + 7) / 8;
-    long long cap = (long long)kNumSMs * 16;
+    long long cap = (long long)num_sms() * 16;
     int grid = (int)(blocks < cap ? blocks : cap);
     if (dtype == REFORM_BF16)
       scan_simt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(

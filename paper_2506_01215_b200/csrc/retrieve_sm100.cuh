@@ -198,7 +198,7 @@ inline int launch_scan_sm100(const void* bank, const void* queries, float* ts, i
       return REFORM_ERR_UNSUPPORTED;
   }
   const int tiles = (int)((N + kScanTileTokens - 1) / kScanTileTokens);
-  int per_b = (kNumSMs + B - 1) / B;
+  int per_b = (num_sms() + B - 1) / B;
   if (per_b > tiles) per_b = tiles;
   if (per_b < 1) per_b = 1;
   cudaFuncSetAttribute(scan_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -87,7 +87,7 @@ inline int launch_rope(const void* src, void* dst, int BH, int d, long long cap,
   const int np = 16 / (int)sizeof(T) / (interleaved ? 2 : 1);
   const long long items = rows * ((d / 2) / np);
   long long blocks = (items + 255) / 256;
-  const long long cap_blocks = (long long)kNumSMs * 16;
+  const long long cap_blocks = (long long)num_sms() * 16;
   const int grid = (int)(blocks < cap_blocks ? blocks : cap_blocks);
   RopeFreq freq;
   for (int i = 0; i < d / 2; ++i) freq.turns[i] = pow(base, -2.0 * i / d) / 6.283185307179586476925;

@@ -53,7 +53,7 @@ inline int launch_gather(const uint4* src, const int32_t* idx, uint4* dst, int B
   while (4 * lanes < vec && lanes < kRowThreads) lanes <<= 1;
   long long rows_per_block = kRowThreads / lanes;
   long long blocks = (total + rows_per_block - 1) / rows_per_block;
-  long long cap = (long long)kNumSMs * 16;
+  long long cap = (long long)num_sms() * 16;
   int grid = (int)(blocks < cap ? blocks : cap);
 #define REFORM_GATHER_CASE(L)                                                                    \
   case L:                                                                                        \
@@ -129,7 +129,7 @@ inline int launch_evict_compact(const void* k_src, const void* v_src, void* k_ds
   while (4 * lanes < vec && lanes < 32) lanes <<= 1;
   long long rows_per_block = kRowThreads / lanes;
   long long blocks = (total + rows_per_block - 1) / rows_per_block;
-  long long cap = (long long)kNumSMs * 8;
+  long long cap = (long long)num_sms() * 8;
   dim3 grid((unsigned)(blocks < cap ? blocks : cap), 2);
 #define REFORM_COMPACT_CASE(L)                                                                   \
   case L:                                                                                        \

@@ -313,8 +313,9 @@ def test_embed_append_matches_oracle(dtype, d, n_slots):
     assert torch.equal(got[:, :11], ref[:, :11]) and torch.equal(got[:, 11 + Lc:], ref[:, 11 + Lc:])
     rows = got[:, 11:11 + Lc].double()
     exact = f64[:, 11:11 + Lc]
-    # fp32 norm (a few ulp), fp32 divide, one rounding to the bank dtype
-    tol = 2.0 ** -8 if dtype == torch.bfloat16 else 4 * 2.0 ** -23
+    # within one unit in the last place of the exact quotient: bf16 banks take fp32 arithmetic and
+    # one rounding, fp32 banks take an fp64 norm and quotient and one rounding
+    tol = 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -23
     assert ((rows - exact).abs() <= tol * exact.abs() + 1e-30).all()
     if dtype == torch.bfloat16:
         same = (got[:, 11:11 + Lc] == ref[:, 11:11 + Lc]).float().mean().item()
@@ -466,28 +467,47 @@ def test_tiny_recurrence_matches_oracle_step_by_step(sink, window):
 
 
 def test_tiny_free_running_pipeline_with_driver():
-    """The binding's driver runs all 8 steps on the GPU alone; the oracle runs
-    them alone; kept positions and final cache agree."""
+    """Config 1 free-running: the binding's driver runs all 8 steps on the GPU alone, the oracle
+    runs them alone.  After every step the kept token positions of every KV head must equal the
+    oracle's, up to swaps between candidates whose oracle scores lie within 1e-4 (relative) of the
+    cutoff, and the carried scores of the kept rows must agree to 1e-3.  A tolerated swap makes the
+    two caches differ from then on, so the comparison ends there and the step, head and score gap
+    of that first divergence are reported."""
+    import warnings
+    from oracle_run import oracle_free_run
     w = synth.WORKLOADS["tiny"]
+    G = w.Hq // w.Hkv
     cache = LayerCache(w.B, w.Hkv, w.d, w.cap, w.budget, w.n_sink, w.n_recent, w.dtype, DEV)
-    ck = torch.zeros(w.B, w.Hkv, w.cap, w.d)
-    cv = torch.zeros_like(ck)
-    cs = torch.zeros(w.B, w.Hkv, w.cap, dtype=torch.float64)
-    n_cache = 0
     out = torch.zeros(w.B, w.Hq, w.Lc, w.d, device=DEV)
-    for step in range(w.steps):
+    pos = torch.zeros(w.B, w.Hkv, w.cap, dtype=torch.int64)            # token position of every GPU cache row
+    for st in oracle_free_run(w):
+        step, n, n_cache = st["step"], st["n"], st["n_cache_before"]
         q, kc, vc = synth.chunk_qkv(w, 0, step)
         cache.write_chunk(kc.to(DEV), vc.to(DEV))
         cache.attend(q.to(DEV), out, w.window)
-        cache.evict()
-        ck[:, :, n_cache:n_cache + w.Lc] = kc
-        cv[:, :, n_cache:n_cache + w.Lc] = vc
-        s_ref = oracle.key_scores(q, ck, n_cache, w.window, score_in=cs, accumulate=True)
-        ref = oracle.evict_topk(ck, cv, s_ref, n_cache + w.Lc, w.budget, w.n_sink, w.n_recent, cap_dst=w.cap)
-        ck, cv, cs, n_cache = ref["k"], ref["v"], ref["score"], ref["n_kept"]
-        same = (cache.k[cache.cur][:, :, :n_cache].cpu() == ck[:, :, :n_cache]).all(-1).float().mean().item()
-        assert same > 0.995, f"step {step}: only {same:.4f} of cache rows agree"
-    assert_scores_close(cache.score[cache.cur][:, :, :n_cache], cs[:, :, :n_cache], 1e-3) if same == 1.0 else None
+        pos[:, :, n_cache:n] = torch.arange(step * w.Lc, (step + 1) * w.Lc)
+        gpu_scores = cache.score[cache.cur][:, :, :n].cpu()
+        assert_scores_close(gpu_scores, st["scores"][:, :, :n], w.window * G / n)
+        n_kept = cache.evict()
+        assert n_kept == st["n_kept"]
+        kept = cache.kept_idx.cpu().long()
+        swaps = 0
+        for h in range(w.Hkv):
+            swaps += assert_index_sets_match(kept[0, h, :n_kept], st["kept_idx"][0, h, :n_kept],
+                                             st["scores"][0, h])
+        pos[:, :, :n_kept] = torch.gather(pos, 2, kept[:, :, :n_kept])
+        if swaps:
+            both = [sorted(set(kept[0, h].tolist()) ^ set(st["kept_idx"][0, h].tolist())) for h in range(w.Hkv)]
+            gap = max(abs(float(st["scores"][0, h][a] - st["scores"][0, h][b]))
+                      for h in range(w.Hkv) for a in both[h] for b in both[h])
+            warnings.warn(f"free run diverged at step {step} by a tolerated swap (score gap {gap:.3e}); "
+                          "later steps are judged by the step-by-step test only")
+            return
+        assert torch.equal(pos[:, :, :n_kept], st["pos"][:, :, :n_kept].long())
+        kd = cache.k[cache.cur][:, :, :n_kept].cpu()
+        assert torch.equal(kd, st["k"][:, :, :n_kept])                 # same rows, bit for bit
+        assert torch.equal(cache.v[cache.cur][:, :, :n_kept].cpu(), st["v"][:, :, :n_kept])
+        assert_scores_close(cache.score[cache.cur][:, :, :n_kept], st["score"][:, :, :n_kept], w.window * G / n)
 
 
 def test_chunk_step_seeded_random_shapes():

@@ -112,6 +112,18 @@ def test_chunk_step_needs_workspace_for_lse():
     assert L.reform_chunk_step(ctypes.byref(_chunk(dtype=7)), None) == R.ERR_UNSUPPORTED
 
 
+def test_chunk_step_size_query_validates_shapes():
+    """The size query answers 0 for arguments the call would reject (it must not divide by a zero
+    head count), and over-large batches are refused up front instead of failing at launch."""
+    L = R.lib()
+    for kw in (dict(Hkv=0), dict(Hq=5), dict(d=48), dict(dtype=7), dict(n_cache=8), dict(struct_size=0)):
+        assert L.reform_chunk_step_workspace_size(ctypes.byref(_chunk(lse=None, **kw))) == 0
+    assert L.reform_chunk_step_workspace_size(ctypes.byref(_chunk(lse=None, Lc=1, cap=1, score_window=1))) > 0
+    assert L.reform_chunk_step(ctypes.byref(_chunk(B=20000, Hq=4)), None) == R.ERR_INVALID_ARG
+    assert L.reform_evict_topk(ctypes.byref(_evict(B=40000)), None) == R.ERR_INVALID_ARG
+    assert L.reform_retrieve_topk(ctypes.byref(_retrieve(B=70000)), None) == R.ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("kw", [
     dict(n_sink=20, n_recent=20), dict(n_keys=200), dict(cap_dst=16), dict(k_dst=FAKE),
     dict(pos_src=FAKE), dict(score_src=None), dict(budget=-1),

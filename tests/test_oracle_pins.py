@@ -457,3 +457,42 @@ def test_rope_scores_depend_on_relative_position_only():
         dots.append((qm.double() * kn.double()).sum().item())
     assert abs(dots[0] - dots[1]) < 1e-4 and abs(dots[0] - dots[2]) < 1e-4
     assert abs(dots[0] - (q.double() * k.double()).sum().item()) > 1e-3   # and it is not the unrotated dot
+
+
+# ------------------------------------------------- recurrence (needle pin)
+
+@pytest.mark.parametrize("accumulate", [True, False])
+def test_tiny_free_run_keeps_every_planted_needle(accumulate):
+    """The Tiny configuration run by the oracle alone for its 8 chunk steps (Alg. 1 ForwardChunk;
+    Sec. 3.1 compression with the first and last 32 rows kept): after every eviction every needle
+    seen so far is still in every KV head's cache.  With per-chunk scores a needle scored among
+    the candidates ranks within the first 2 x n_needles of them (only other needles and a few lucky
+    keys out-score a +4 logit); with accumulated scores the survivors of earlier steps carry
+    several chunks of mass, so the claim there is the weaker one that the needle ranks inside the
+    kept set.  The planted keys are heavy by construction, so a selection that dropped one would
+    be wrong by the definition itself."""
+    from oracle_run import oracle_free_run
+    from paper_2506_01215_b200 import synth
+    w = synth.WORKLOADS["tiny"]
+    needles = synth.needle_positions(w)
+    assert len(set(needles)) == w.n_needles == 8
+    m = w.budget - w.n_sink - w.n_recent
+    steps = 0
+    for st in oracle_free_run(w, accumulate=accumulate):
+        steps += 1
+        seen = [p for p in needles if p < (st["step"] + 1) * w.Lc]
+        assert st["n_kept"] == w.budget
+        for h in range(w.Hkv):
+            kept = st["pos"][0, h, :w.budget]
+            assert (kept[1:] > kept[:-1]).all()                           # order preserved
+            assert set(seen) <= set(kept.tolist()), f"needle lost in head {h}, step {st['step']}"
+            before = st["pos_before"][0, h, :st["n"]].tolist()
+            sc = st["scores"][0, h, :st["n"]]
+            cand = sc[w.n_sink:st["n"] - w.n_recent]
+            for p in seen:
+                r = before.index(p)
+                if w.n_sink <= r < st["n"] - w.n_recent:                  # scored as a candidate
+                    rank = int((cand > sc[r]).sum())
+                    bound = m if accumulate else 2 * w.n_needles
+                    assert rank < bound, f"needle {p} ranks {rank} of {cand.numel()} candidates"
+    assert steps == w.steps == 8

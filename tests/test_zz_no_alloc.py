@@ -11,6 +11,7 @@ import ctypes
 import pytest
 import torch
 
+import oracle
 import paper_2506_01215_b200 as R
 
 DEV = "cuda"
@@ -51,6 +52,12 @@ def test_static_entry_point_matches_regular_one_on_two_calls_in_a_row():
         assert n_got == n_ref == budget
         for a, b in zip(got, ref):
             assert torch.equal(a, b)      # integer, byte and index work: bit-exact
+        # and both equal the oracle's full sort
+        o = oracle.evict_topk(k.cpu(), v.cpu(), sc.cpu(), n_keys, budget, sink, recent, cap_dst=budget,
+                              pos_src=pos.cpu())
+        assert torch.equal(got[4].cpu(), o["kept_idx"])
+        assert torch.equal(got[0].cpu().view(torch.uint8), o["k"].view(torch.uint8))
+        assert torch.equal(got[2].cpu().double(), o["score"]) and torch.equal(got[3].cpu(), o["pos"])
     # and once more without the optional kept-index output (the list then lives in the scratch)
     seed, B, Hkv, n_keys, d, budget, sink, recent, dtype = cases[0]
     k, v, sc, pos = _inputs(seed, B, Hkv, n_keys, d, dtype)
@@ -61,6 +68,28 @@ def test_static_entry_point_matches_regular_one_on_two_calls_in_a_row():
     torch.cuda.synchronize()
     for a, b in zip(got[:3], ref[:3]):
         assert torch.equal(a, b)
+
+
+@pytest.mark.gpu
+def test_static_entry_point_at_its_documented_limits():
+    """The largest problem the built-in scratch takes: 32 segments x 65,536 keys, budget 16,384, no
+    kept-index output (so the list itself lives in the scratch, which this case fills almost to
+    its last byte) -- more selection blocks than can be resident at once, so the selection runs as
+    one launch per pass.  Twice back to back on different inputs, each against the oracle."""
+    B, Hkv, n_keys, d, budget = 4, 8, R.EVICT_STATIC_MAX_KEYS, 64, R.EVICT_STATIC_MAX_BUDGET
+    assert B * Hkv == R.EVICT_STATIC_MAX_SEGS
+    for seed in (21, 22):
+        k, v, sc, pos = _inputs(seed, B, Hkv, n_keys - 3, d, torch.bfloat16)     # cap = n_keys exactly
+        got = _outputs(B, Hkv, budget, d, torch.bfloat16)
+        n = R.evict_topk_static(k, v, sc, got[0], got[1], got[2], n_keys, budget, 256, 256,
+                                pos_src=pos, pos_dst=got[3])
+        torch.cuda.synchronize()
+        assert n == budget and R.device_error() == 0
+        o = oracle.evict_topk(k.cpu(), v.cpu(), sc.cpu(), n_keys, budget, 256, 256, cap_dst=budget,
+                              pos_src=pos.cpu())
+        assert torch.equal(got[0].cpu().view(torch.uint8), o["k"].view(torch.uint8))
+        assert torch.equal(got[1].cpu().view(torch.uint8), o["v"].view(torch.uint8))
+        assert torch.equal(got[2].cpu().double(), o["score"]) and torch.equal(got[3].cpu(), o["pos"])
 
 
 @pytest.mark.gpu
