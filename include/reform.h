@@ -209,6 +209,27 @@ int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream);
 int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t stream);
 
 /* ------------------------------------------------------------------------
+ * reform_debug_evict_wait_expiry -- diagnostic, no counterpart in the paper.
+ * The kernels of this library never wait without a limit: a block that waits
+ * for another block, for a copy or for the tensor cores gives up after a
+ * bounded time, raises REFORM_DEV_TIMEOUT and lets the launch wind down with
+ * the context intact.  This entry point lets a test see that happen without
+ * faulting anything: it runs reform_evict_topk's one-launch form with the
+ * hand-off waits limited to wait_cycles SM clock cycles and with every
+ * selection block waiting for one block more than the launch has -- a flag
+ * that nothing ever sets.  Every block's first wait therefore runs out; the
+ * kernel returns, REFORM_DEV_TIMEOUT is set in *p->dev_status and in the
+ * per-device error word, and the outputs are unspecified.  The call after it
+ * behaves as if this one had not happened.
+ * Arguments as for reform_evict_topk.  wait_cycles in (0, 400,000,000].
+ * REFORM_ERR_UNSUPPORTED if the shape would not take the one-launch form
+ * (nothing to choose, 48 or more short segments, more blocks than fit the
+ * device at once).
+ * ------------------------------------------------------------------------ */
+int reform_debug_evict_wait_expiry(const reform_evict_params* p, long long wait_cycles,
+                                   reform_stream_t stream);
+
+/* ------------------------------------------------------------------------
  * reform_embed_append -- Sec. 3.2 "Combining multiple heads":
  *   e_comb = concat_i ( e_i / ||e_i|| ).
  *

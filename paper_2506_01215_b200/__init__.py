@@ -82,7 +82,8 @@ class RopeParams(ctypes.Structure):
 
 EXPORTS = (
     "reform_chunk_step", "reform_chunk_step_workspace_size", "reform_evict_topk",
-    "reform_evict_topk_workspace_size", "reform_evict_topk_static", "reform_embed_append", "reform_retrieve_topk",
+    "reform_evict_topk_workspace_size", "reform_evict_topk_static", "reform_debug_evict_wait_expiry",
+    "reform_embed_append", "reform_retrieve_topk",
     "reform_retrieve_topk_workspace_size", "reform_gather", "reform_rope", "reform_status_string",
     "reform_last_cuda_error", "reform_device_error", "reform_version", "reform_kernel_launch_count",
 )
@@ -116,6 +117,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name + "_workspace_size").restype = _sz
         L.reform_evict_topk_static.argtypes = [ctypes.POINTER(EvictParams), _vp]
         L.reform_evict_topk_static.restype = ctypes.c_int
+        L.reform_debug_evict_wait_expiry.argtypes = [ctypes.POINTER(EvictParams), ctypes.c_longlong, _vp]
+        L.reform_debug_evict_wait_expiry.restype = ctypes.c_int
         L.reform_embed_append.argtypes = [ctypes.POINTER(EmbedParams), _vp]
         L.reform_embed_append.restype = ctypes.c_int
         L.reform_gather.argtypes = [ctypes.POINTER(GatherParams), _vp]
@@ -225,6 +228,23 @@ def evict_topk(k_src, v_src, score_src, k_dst, v_dst, score_dst, n_keys: int, bu
         p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel() * ws.element_size()
     _check("reform_evict_topk", lib().reform_evict_topk(ctypes.byref(p), _stream(stream)))
     return n_kept.value
+
+
+def debug_evict_wait_expiry(k_src, v_src, score_src, k_dst, v_dst, score_dst, n_keys: int, budget: int,
+                            n_sink: int, n_recent: int, wait_cycles: int, dev_status, *, stream=None):
+    """reform_debug_evict_wait_expiry: the eviction's one-launch form with its hand-off waits
+    limited to wait_cycles and waiting for a flag that nothing sets; REFORM_DEV_TIMEOUT lands in
+    dev_status (a device int32 tensor) and in the per-device error word.  Outputs are unspecified."""
+    B, Hkv, cap_src, d = k_src.shape
+    p = EvictParams(ctypes.sizeof(EvictParams), _dtype_code(k_src), B, Hkv, d, int(n_keys), cap_src,
+                    k_dst.shape[2], int(budget), int(n_sink), int(n_recent), _ptr(k_src), _ptr(v_src),
+                    _ptr(score_src), None, _ptr(k_dst), _ptr(v_dst), _ptr(score_dst), None, None, None,
+                    None, 0, _ptr(dev_status))
+    need = lib().reform_evict_topk_workspace_size(ctypes.byref(p))
+    ws = workspace(need, k_src.device)
+    p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel() * ws.element_size()
+    _check("reform_debug_evict_wait_expiry",
+           lib().reform_debug_evict_wait_expiry(ctypes.byref(p), int(wait_cycles), _stream(stream)))
 
 
 def evict_topk_static(k_src, v_src, score_src, k_dst, v_dst, score_dst, n_keys: int, budget: int,

@@ -2,12 +2,15 @@
 // carving and kernel dispatch.  Every entry point either returns an error
 // before launching anything or enqueues its kernels on the caller's stream.
 #include <atomic>
+#include <chrono>
+#include <random>
 
 #include "common.cuh"
 #include "rows.cuh"
 #include "embed.cuh"
 #include "rope.cuh"
 #include "select.cuh"
+#include "evict_fused.cuh"
 #include "retrieve.cuh"
 #include "chunk_simt.cuh"
 #if !defined(REFORM_NO_SM100) && !__has_include("chunk_sm100.cuh")
@@ -23,6 +26,24 @@ namespace reform {
 thread_local int g_last_cuda_error = 0;
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+unsigned long long next_epoch() {
+  static const unsigned long long salt = [] {
+    unsigned long long x = (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count();
+    try {
+      std::random_device rd;
+      x ^= ((unsigned long long)rd() << 32) ^ rd();
+    } catch (...) {
+    }
+    return x;
+  }();
+  static std::atomic<unsigned long long> counter{1};
+  unsigned long long e;
+  do {
+    e = (salt + counter.fetch_add(1, std::memory_order_relaxed)) << 3;
+  } while (e == 0);
+  return e;
+}
 
 static size_t elem_size(int dtype) { return dtype == REFORM_F32 ? 4 : 2; }
 static bool dtype_ok(int dtype) { return dtype == REFORM_F32 || dtype == REFORM_BF16; }
@@ -156,50 +177,116 @@ static size_t evict_kept_bytes(const reform_evict_params* p) {
   return align_up(sizeof(int32_t) * (size_t)p->B * p->Hkv * (p->budget > 0 ? p->budget : 1), 256);
 }
 
-size_t reform_evict_topk_workspace_size(const reform_evict_params* p) {
-  if (!p || p->struct_size != sizeof(reform_evict_params)) return 0;
-  if (p->B <= 0 || p->Hkv <= 0) return 0;
-  int segs = p->B * p->Hkv;
-  return sel_layout(segs, p->n_keys).total + (p->kept_idx ? 0 : evict_kept_bytes(p));
+// Smallest workspace with which the call can run at all (the per-pass selection path).
+static size_t evict_workspace_min(const reform_evict_params* p) {
+  return sel_layout(p->B * p->Hkv, p->n_keys).total + (p->kept_idx ? 0 : evict_kept_bytes(p));
 }
 
-int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream) {
-  int rc = validate_evict(p);
-  if (rc != REFORM_OK) return rc;
+size_t reform_evict_topk_workspace_size(const reform_evict_params* p) {
+  if (!p || p->struct_size != sizeof(reform_evict_params)) return 0;
+  if (p->B <= 0 || p->Hkv <= 0 || p->n_keys < 0) return 0;
+  const size_t fused = evict_fused_layout(p->B * p->Hkv, p->n_keys).total + (p->kept_idx ? 0 : evict_kept_bytes(p));
+  const size_t basic = evict_workspace_min(p);
+  return fused > basic ? fused : basic;
+}
+
+// need: the workspace size the entry point insists on.  wait_cycles / expect_extra: limits of the
+// hand-off waits of the one-launch form (diagnostic entry point; kEvWaitCycles and 0 otherwise).
+static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need, long long wait_cycles,
+                     int expect_extra) {
   const int n_kept = p->n_keys < p->budget ? p->n_keys : p->budget;
   if (p->n_kept_host) *p->n_kept_host = n_kept;
   const int segs = p->B * p->Hkv;
   if (segs == 0 || n_kept == 0) return REFORM_OK;
-  size_t need = reform_evict_topk_workspace_size(p);
   if (!p->workspace || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
     return REFORM_ERR_WORKSPACE;
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   char* ws = reinterpret_cast<char*>(p->workspace);
+  int lo, hi, m;
+  if (p->n_keys <= p->budget) {  // keep everything: all rows are "forced"
+    lo = hi = p->n_keys;
+    m = 0;
+  } else {
+    lo = p->n_sink;
+    hi = p->n_keys - p->n_recent;
+    m = p->budget - p->n_sink - p->n_recent;
+  }
+  const int row_bytes = (int)(p->d * elem_size(p->dtype));
+  const size_t kept_bytes = p->kept_idx ? 0 : evict_kept_bytes(p);
+  const bool many_short = p->n_keys <= kSelBlockMaxN && segs >= kSelBlockMinSegs;  // one block per segment wins
+  if (!many_short && evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes)) {
+    // one cooperative launch: selection with two hand-offs, then the compaction
+    const EvictFusedLayout F = evict_fused_layout(segs, p->n_keys);
+    EvictFusedArgs a;
+    a.vals = p->score_src;
+    a.stride = p->cap_src;
+    a.n = p->n_keys;
+    a.lo = lo;
+    a.hi = hi;
+    a.m = m;
+    a.out = p->kept_idx ? p->kept_idx : reinterpret_cast<int32_t*>(ws + F.total);
+    a.out_stride = p->budget;
+    a.segs = segs;
+    a.nb = F.nb;
+    a.slices = reinterpret_cast<uint32_t*>(ws + F.slices);
+    a.cand = reinterpret_cast<uint32_t*>(ws + F.cand);
+    a.flags = reinterpret_cast<unsigned long long*>(ws + F.flags);
+    a.expect_extra = expect_extra;
+    a.epoch = next_epoch();
+    a.wait_cycles = wait_cycles;
+    a.k_src = (const uint4*)p->k_src;
+    a.v_src = (const uint4*)p->v_src;
+    a.k_dst = (uint4*)p->k_dst;
+    a.v_dst = (uint4*)p->v_dst;
+    a.score_src = p->score_src;
+    a.score_dst = p->score_dst;
+    a.pos_src = p->pos_src;
+    a.pos_dst = p->pos_dst;
+    a.n_kept = n_kept;
+    a.cap_src = p->cap_src;
+    a.cap_dst = p->cap_dst;
+    a.vec = row_bytes / 16;
+    a.dev_status = p->dev_status;
+    return launch_evict_fused(a, st);
+  }
   SelLayout L = sel_layout(segs, p->n_keys);
   int32_t* kept = p->kept_idx ? p->kept_idx : reinterpret_cast<int32_t*>(ws + L.total);
   SelArgs a;
   a.vals = p->score_src;
   a.stride = p->cap_src;
   a.n = p->n_keys;
-  if (p->n_keys <= p->budget) {  // keep everything: all rows are "forced"
-    a.lo = a.hi = p->n_keys;
-    a.m = 0;
-  } else {
-    a.lo = p->n_sink;
-    a.hi = p->n_keys - p->n_recent;
-    a.m = p->budget - p->n_sink - p->n_recent;
-  }
+  a.lo = lo;
+  a.hi = hi;
+  a.m = m;
   a.out = kept;
   a.out_stride = p->budget;
   a.state = reinterpret_cast<SelState*>(ws + L.state);
   a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
   a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
   a.blocks_per_seg = L.blocks_per_seg;
-  rc = launch_select(a, segs, nullptr, nullptr, 0, ws, L, p->dev_status, st);
+  int rc = launch_select(a, segs, nullptr, nullptr, 0, ws, L, p->dev_status, st);
   if (rc != REFORM_OK) return rc;
   return launch_evict_compact(p->k_src, p->v_src, p->k_dst, p->v_dst, p->score_src, p->score_dst,
                               p->pos_src, p->pos_dst, kept, p->budget, segs, n_kept, p->cap_src,
-                              p->cap_dst, (int)(p->d * elem_size(p->dtype)), st);
+                              p->cap_dst, row_bytes, st);
+}
+
+int reform_evict_topk(const reform_evict_params* p, reform_stream_t stream) {
+  int rc = validate_evict(p);
+  if (rc != REFORM_OK) return rc;
+  return evict_run(p, reinterpret_cast<cudaStream_t>(stream), reform_evict_topk_workspace_size(p), kEvWaitCycles, 0);
+}
+
+int reform_debug_evict_wait_expiry(const reform_evict_params* p, long long wait_cycles, reform_stream_t stream) {
+  int rc = validate_evict(p);
+  if (rc != REFORM_OK) return rc;
+  if (wait_cycles <= 0 || wait_cycles > kEvWaitCycles) return REFORM_ERR_INVALID_ARG;
+  const int segs = p->B * p->Hkv;
+  const size_t kept_bytes = p->kept_idx ? 0 : evict_kept_bytes(p);
+  const bool many_short = p->n_keys <= kSelBlockMaxN && segs >= kSelBlockMinSegs;
+  if (segs == 0 || p->n_keys <= p->budget || p->budget == p->n_sink + p->n_recent || many_short ||
+      !evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes))
+    return REFORM_ERR_UNSUPPORTED;   // only the one-launch form has hand-off waits to run out
+  return evict_run(p, reinterpret_cast<cudaStream_t>(stream), reform_evict_topk_workspace_size(p), wait_cycles, 1);
 }
 
 /* ------------------------------------------ evict without a workspace */
@@ -240,13 +327,15 @@ int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t strea
   reform_evict_params q = *p;
   q.workspace = nullptr;
   q.workspace_bytes = 0;
-  if (reform_evict_topk_workspace_size(&q) > REFORM_EVICT_STATIC_BYTES) return REFORM_ERR_TOO_LARGE;
+  const size_t need = evict_workspace_min(&q);
+  if (need > REFORM_EVICT_STATIC_BYTES) return REFORM_ERR_TOO_LARGE;
   void* scratch = nullptr;
   rc = evict_static_scratch(&scratch);
   if (rc != REFORM_OK) return rc;
   q.workspace = scratch;
   q.workspace_bytes = REFORM_EVICT_STATIC_BYTES;
-  return reform_evict_topk(&q, stream);
+  // the one-launch form is taken when its (larger) layout fits the array too
+  return evict_run(&q, reinterpret_cast<cudaStream_t>(stream), need, kEvWaitCycles, 0);
 }
 
 /* ---------------------------------------------------------------- embed */

@@ -278,6 +278,54 @@ def test_retrieve_many_sequences_multi_launch_path():
         assert_index_sets_match(idx[b].cpu(), ref["idx"][b], ref["pooled"][b])
 
 
+def test_evict_all_scores_equal_and_two_level_ties():
+    """Degenerate score distributions for the one-launch selection: every candidate in one
+    histogram bin (all scores equal: the kept middle rows are the lowest indices), and scores that
+    agree in their leading bits and differ only in the last ones."""
+    g = torch.Generator().manual_seed(3)
+    B, Hkv, n, d, budget = 1, 3, 13000, 8, 3000
+    k = torch.randn(B, Hkv, n, d, generator=g)
+    for sc in (torch.full((B, Hkv, n), 0.37),
+               1.0 + torch.randint(0, 50, (B, Hkv, n), generator=g).float() * 2.0 ** -23,
+               torch.zeros(B, Hkv, n)):
+        ref = oracle.evict_topk(k, k, sc, n, budget, 7, 9, cap_dst=budget)
+        kd = torch.zeros(B, Hkv, budget, d, device=DEV)
+        vd, sd = torch.zeros_like(kd), torch.zeros(B, Hkv, budget, device=DEV)
+        kept = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV)
+        R.evict_topk(k.to(DEV), k.to(DEV).clone(), sc.to(DEV), kd, vd, sd, n, budget, 7, 9, kept_idx=kept)
+        assert torch.equal(kept.cpu(), ref["kept_idx"])
+        assert torch.equal(kd.cpu(), ref["k"]) and torch.equal(sd.cpu().double(), ref["score"])
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """Failure detection without a fault: the eviction's one-launch form is made to wait, for
+    about a millisecond, on a flag that nothing sets.  Every block gives up, the kernel returns,
+    REFORM_DEV_TIMEOUT shows in the caller's status word and in the library's per-device word,
+    and the next ordinary call on the same workspace is bit-exact against the oracle."""
+    g = torch.Generator().manual_seed(17)
+    B, Hkv, n, d, budget = 1, 4, 9000, 64, 2048
+    k = torch.randn(B, Hkv, n, d, generator=g).to(torch.bfloat16)
+    v = torch.randn(B, Hkv, n, d, generator=g).to(torch.bfloat16)
+    sc = torch.rand(B, Hkv, n, generator=g)
+    kd = torch.zeros(B, Hkv, budget, d, dtype=torch.bfloat16, device=DEV)
+    vd, sd = torch.zeros_like(kd), torch.zeros(B, Hkv, budget, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    assert R.device_error() == 0
+    R.debug_evict_wait_expiry(k.to(DEV), v.to(DEV), sc.to(DEV), kd, vd, sd, n, budget, 64, 64,
+                              wait_cycles=2_000_000, dev_status=status)
+    torch.cuda.synchronize()                                  # returns: nothing hangs, nothing faults
+    assert status.item() == R.DEV_TIMEOUT
+    assert R.device_error() == R.DEV_TIMEOUT                  # kept by the library too; reading clears it
+    assert R.device_error() == 0
+    kept = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV)
+    R.evict_topk(k.to(DEV), v.to(DEV), sc.to(DEV), kd, vd, sd, n, budget, 64, 64, kept_idx=kept)
+    ref = oracle.evict_topk(k, v, sc, n, budget, 64, 64, cap_dst=budget)
+    assert torch.equal(kept.cpu(), ref["kept_idx"])
+    assert torch.equal(kd.cpu().view(torch.int16), ref["k"].view(torch.int16))
+    assert torch.equal(vd.cpu().view(torch.int16), ref["v"].view(torch.int16))
+    assert R.device_error() == 0
+
+
 def test_evict_without_optional_outputs():
     g = torch.Generator().manual_seed(1)
     k = torch.randn(1, 2, 600, 64, generator=g)
