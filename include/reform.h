@@ -77,8 +77,13 @@ enum {
 enum {
   REFORM_SCORE_ACCUMULATE = 1u, /* score[j] += carried score for cache rows j < n_cache */
   REFORM_NO_SCORE = 2u,         /* skip the key-score pass (plain prefill attention) */
-  REFORM_FORCE_SIMT = 4u        /* use the CUDA-core kernels even where a tensor-core path exists */
+  REFORM_FORCE_SIMT = 4u,       /* use the CUDA-core kernels even where a tensor-core path exists */
+  REFORM_ROPE = 8u,             /* q and k are un-rotated: apply the rotary embedding inside the call */
+  REFORM_ROPE_INTERLEAVED = 16u /* with REFORM_ROPE: pairs are (x[2i], x[2i+1]) instead of (x[i], x[i+d/2]) */
 };
+
+/* pooling of the token scores in reform_retrieve_topk */
+enum { REFORM_POOL_MAX = 0, REFORM_POOL_MEAN = 1 };
 
 /* kinds of state a context-embedding slot can come from */
 enum { REFORM_STATE_Q = 0, REFORM_STATE_K = 1, REFORM_STATE_V = 2 };
@@ -108,6 +113,17 @@ enum { REFORM_STATE_Q = 0, REFORM_STATE_K = 1, REFORM_STATE_V = 2 };
  * its partial results even when lse is given: always size the workspace with
  * reform_chunk_step_workspace_size().
  * softmax_scale 0 means 1/sqrt(d).  score_window in [1, Lc].
+ *
+ * REFORM_ROPE (Sec. 3.1, position re-assignment after compression): the cache
+ * keeps un-rotated keys because every eviction renumbers its rows, so q and k
+ * are passed un-rotated and the call rotates them at the ids of the moment --
+ * row r of [cache ; chunk] at position r, chunk query i at n_cache + i, angle
+ * pos * rope_theta^(-2 pair / d) as in reform_rope -- and computes out, lse and
+ * score from the rotated operands.  q and k themselves are not modified.  On
+ * the tensor-core path each query tile is rotated in shared memory right after
+ * it is loaded; the keys, which every block re-reads, are rotated once per call
+ * into the workspace (as are the score window's query rows), so size the
+ * workspace with reform_chunk_step_workspace_size().  rope_theta 0 means 10000.
  * ------------------------------------------------------------------------ */
 typedef struct reform_chunk_params {
   size_t struct_size;
@@ -117,6 +133,7 @@ typedef struct reform_chunk_params {
   int32_t score_window;
   float softmax_scale;
   uint32_t flags;
+  float rope_theta;
   const void* q;
   const void* k;
   const void* v;
@@ -282,6 +299,12 @@ int reform_embed_append(const reform_embed_params* p, reform_stream_t stream);
  *   selected  = tokens [0, n_keep_head) and [N - n_keep_tail, N), plus the
  *               k - n_keep_head - n_keep_tail other tokens with the largest
  *               pooled score (ties to the lower index), ascending.
+ * With pool_mode == REFORM_POOL_MEAN, pooled[t] is instead the mean of ts over
+ * the same clipped window (divided by the number of tokens in it): the
+ * smoothing the paper applies when it ranks heads (Appendix, detailed head
+ * selection, Step 3: mean over a token and its 20 neighbours is pool_window =
+ * 21).  The window is summed directly, so this mode costs O(pool_window) per
+ * token.
  * Bank rows are stored per-head normalised (reform_embed_append), so the
  * cosine of Sec. 3.2 is this dot product with scale = 1 / n_slots.
  *
@@ -300,6 +323,7 @@ typedef struct reform_retrieve_params {
   int32_t pool_window;
   int32_t n_keep_head, n_keep_tail;
   int32_t k;
+  int32_t pool_mode; /* REFORM_POOL_MAX or REFORM_POOL_MEAN */
   const void* bank;
   const void* queries;
   int32_t* idx_out;

@@ -154,8 +154,10 @@ def embed_append(bank, token_offset, sel, q_state=None, k_state=None, v_state=No
     return f64
 
 
-def retrieve_topk(bank, queries, N, k, scale=1.0, pool_window=1, n_keep_head=0, n_keep_tail=0):
-    """Returns dict(idx [B,n_out] int32 ascending, ts [B,N], pooled [B,N] fp64)."""
+def retrieve_topk(bank, queries, N, k, scale=1.0, pool_window=1, n_keep_head=0, n_keep_tail=0,
+                  pool_mode="max"):
+    """Returns dict(idx [B,n_out] int32 ascending, ts [B,N], pooled [B,N] fp64).  pool_mode "max"
+    (Sec. 3.3) or "mean" (the smoothing of the head-ranking procedure)."""
     B, N_cap, E = bank.shape
     nq = queries.shape[1]
     idx = torch.full((B, k), -1, dtype=torch.int32)
@@ -164,7 +166,7 @@ def retrieve_topk(bank, queries, N, k, scale=1.0, pool_window=1, n_keep_head=0, 
     rc = _load().oracle_retrieve_topk(
         _dt(bank), B, ctypes.c_longlong(int(N)), ctypes.c_longlong(N_cap), E, _p(bank), nq,
         _p(queries), ctypes.c_double(scale), int(pool_window), int(n_keep_head), int(n_keep_tail),
-        int(k), _p(idx), _p(ts), _p(pooled))
+        int(k), _p(idx), _p(ts), _p(pooled), {"max": 0, "mean": 1}[pool_mode])
     if rc < 0:
         raise ValueError("oracle_retrieve_topk: bad arguments")
     return dict(idx=idx[:, :rc].contiguous(), ts=ts, pooled=pooled, n_out=rc)

@@ -346,15 +346,20 @@ int oracle_embed_append(int dtype, int B, int Lc, int d, int Hq, int Hkv, const 
 
 // Token selection.  sim[q][t] = scale * <queries[q], bank[t]>; ts[t] = max_q
 // sim; pooled[t] = max of ts over [t-r, t+r] clipped to [0, N), r =
-// (pool_window-1)/2; tokens [0, n_keep_head) and [N-n_keep_tail, N) are
+// (pool_window-1)/2 (Sec. 3.3), or with pool_mode == 1 the mean of ts over that
+// clipped window (the smoothing used when heads are ranked, Appendix "Detailed
+// head selection process", Step 3: the window is the token and its neighbours,
+// and at the ends the mean runs over the tokens that exist);
+// tokens [0, n_keep_head) and [N-n_keep_tail, N) are
 // always selected; the remaining k - forced come from the other tokens in
 // order (pooled desc, index asc) by a full sort; output ascending.
 // Returns the number selected (min(k, N)) or < 0 on bad arguments.
 int oracle_retrieve_topk(int dtype, int B, long long N, long long N_cap, int E, const void* bank,
                          int nq, const void* queries, double scale, int pool_window,
                          int n_keep_head, int n_keep_tail, int k, int32_t* idx_out,
-                         double* ts_out, double* pooled_out) {
+                         double* ts_out, double* pooled_out, int pool_mode) {
   if (N > N_cap || nq < 1 || pool_window < 1 || pool_window % 2 == 0) return -1;
+  if (pool_mode != 0 && pool_mode != 1) return -1;
   if (n_keep_head < 0 || n_keep_tail < 0 || n_keep_head + n_keep_tail > k) return -1;
   int n_out = (int)std::min<long long>(k, N);
   int r = (pool_window - 1) / 2;
@@ -375,9 +380,15 @@ int oracle_retrieve_topk(int dtype, int B, long long N, long long N_cap, int E, 
     parallel_for((size_t)N, [&](size_t t) {
       long long lo = std::max<long long>(0, (long long)t - r);
       long long hi = std::min<long long>(N - 1, (long long)t + r);
-      double best = ts[lo];
-      for (long long u = lo + 1; u <= hi; ++u) best = std::max(best, ts[u]);
-      pooled[t] = best;
+      if (pool_mode == 0) {
+        double best = ts[lo];
+        for (long long u = lo + 1; u <= hi; ++u) best = std::max(best, ts[u]);
+        pooled[t] = best;
+      } else {
+        double sum = 0.0;
+        for (long long u = lo; u <= hi; ++u) sum += ts[u];
+        pooled[t] = sum / (double)(hi - lo + 1);
+      }
     });
     if (ts_out) std::memcpy(ts_out + (size_t)b * N, ts.data(), sizeof(double) * (size_t)N);
     if (pooled_out) std::memcpy(pooled_out + (size_t)b * N, pooled.data(), sizeof(double) * (size_t)N);

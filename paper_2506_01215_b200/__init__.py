@@ -19,8 +19,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libreform.so")
 
 F32, BF16 = 0, 1
-SCORE_ACCUMULATE, NO_SCORE, FORCE_SIMT = 1, 2, 4
+SCORE_ACCUMULATE, NO_SCORE, FORCE_SIMT, ROPE, ROPE_INTERLEAVED = 1, 2, 4, 8, 16
 STATE_Q, STATE_K, STATE_V = 0, 1, 2
+POOL_MAX, POOL_MEAN = 0, 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5
 EVICT_STATIC_MAX_SEGS, EVICT_STATIC_MAX_KEYS, EVICT_STATIC_MAX_BUDGET = 32, 65536, 16384
 DEV_TIMEOUT, DEV_BAD_INDEX = 1, 2
@@ -33,7 +34,7 @@ _vp, _i32, _i64, _f32, _u32, _sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_in
 class ChunkParams(ctypes.Structure):
     _fields_ = [("struct_size", _sz), ("dtype", _i32), ("B", _i32), ("Hq", _i32), ("Hkv", _i32),
                 ("d", _i32), ("Lc", _i32), ("n_cache", _i32), ("cap", _i32), ("score_window", _i32),
-                ("softmax_scale", _f32), ("flags", _u32), ("q", _vp), ("k", _vp), ("v", _vp),
+                ("softmax_scale", _f32), ("flags", _u32), ("rope_theta", _f32), ("q", _vp), ("k", _vp), ("v", _vp),
                 ("out", _vp), ("lse", _vp), ("score", _vp), ("workspace", _vp),
                 ("workspace_bytes", _sz), ("dev_status", _vp)]
 
@@ -62,7 +63,7 @@ class EmbedParams(ctypes.Structure):
 class RetrieveParams(ctypes.Structure):
     _fields_ = [("struct_size", _sz), ("dtype", _i32), ("B", _i32), ("N", _i64), ("N_cap", _i64),
                 ("E", _i32), ("nq", _i32), ("scale", _f32), ("pool_window", _i32),
-                ("n_keep_head", _i32), ("n_keep_tail", _i32), ("k", _i32), ("bank", _vp),
+                ("n_keep_head", _i32), ("n_keep_tail", _i32), ("k", _i32), ("pool_mode", _i32), ("bank", _vp),
                 ("queries", _vp), ("idx_out", _vp), ("token_score_out", _vp),
                 ("pooled_score_out", _vp), ("workspace", _vp), ("workspace_bytes", _sz),
                 ("dev_status", _vp)]
@@ -196,13 +197,15 @@ def _check(fn: str, rc: int):
 
 
 def chunk_step(q, k, v, out, score, n_cache: int, score_window: int, *, lse=None,
-               softmax_scale: float = 0.0, flags: int = 0, ws=None, dev_status=None, stream=None):
+               softmax_scale: float = 0.0, flags: int = 0, rope_theta: float = 0.0, ws=None, dev_status=None,
+               stream=None):
     """reform_chunk_step: q [B,Hq,Lc,d], k/v [B,Hkv,cap,d], out like q,
-    score [B,Hkv,cap] fp32 (in/out), lse [B,Hq,Lc] fp32 (optional)."""
+    score [B,Hkv,cap] fp32 (in/out), lse [B,Hq,Lc] fp32 (optional).  With ROPE in flags, q and k
+    are un-rotated and the call applies the rotary embedding (base rope_theta) itself."""
     B, Hq, Lc, d = q.shape
     _, Hkv, cap, _ = k.shape
     p = ChunkParams(ctypes.sizeof(ChunkParams), _dtype_code(q), B, Hq, Hkv, d, Lc, int(n_cache), cap,
-                    int(score_window), float(softmax_scale), int(flags), _ptr(q), _ptr(k), _ptr(v),
+                    int(score_window), float(softmax_scale), int(flags), float(rope_theta), _ptr(q), _ptr(k), _ptr(v),
                     _ptr(out), _ptr(lse), _ptr(score), None, 0, _ptr(dev_status))
     need = lib().reform_chunk_step_workspace_size(ctypes.byref(p))
     ws = ws if ws is not None else workspace(need, q.device)
@@ -284,13 +287,14 @@ def embed_append(bank, token_offset: int, sel: Sequence[Tuple[int, int, int]], *
 
 def retrieve_topk(bank, queries, N: int, k: int, idx_out, *, scale: float = 1.0,
                   pool_window: int = 1, n_keep_head: int = 0, n_keep_tail: int = 0,
-                  token_score_out=None, pooled_score_out=None, ws=None, stream=None) -> int:
+                  token_score_out=None, pooled_score_out=None, pool_mode: int = POOL_MAX, ws=None,
+                  stream=None) -> int:
     """reform_retrieve_topk; returns n_out = min(k, N)."""
     B, N_cap, E = bank.shape
     nq = queries.shape[1]
     p = RetrieveParams(ctypes.sizeof(RetrieveParams), _dtype_code(bank), B, int(N), N_cap, E, nq,
                        float(scale), int(pool_window), int(n_keep_head), int(n_keep_tail), int(k),
-                       _ptr(bank), _ptr(queries), _ptr(idx_out), _ptr(token_score_out),
+                       int(pool_mode), _ptr(bank), _ptr(queries), _ptr(idx_out), _ptr(token_score_out),
                        _ptr(pooled_score_out), None, 0, None)
     need = lib().reform_retrieve_topk_workspace_size(ctypes.byref(p))
     ws = ws if ws is not None else workspace(need, bank.device)

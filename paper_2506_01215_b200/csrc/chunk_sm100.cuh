@@ -26,6 +26,7 @@
 
 #include "common.cuh"
 #include "chunk_simt.cuh"
+#include "rope.cuh"
 #include "sm100_ptx.cuh"
 
 namespace reform {
@@ -107,11 +108,66 @@ __device__ __forceinline__ Attn2Tile attn2_tile(int u, int U, int G, int n_qt, i
   return t;
 }
 
+// Rotary embedding of one row of a query tile in shared memory (Sec. 3.1: chunk row i sits at
+// position n_cache + i once the cache rows have been renumbered).  The tile is two boxes of 64
+// columns, 128 bytes per row, 16-byte chunks XOR-swizzled by (row & 7); column c of box 0 and
+// column c of box 1 share an offset, which is where the two halves of a rotate-half pair live.
+// tab: the row's 64 (cos, sin) pairs.
+__device__ __forceinline__ void rope_rotate_q_row(uint8_t* tile, int r, const float2* __restrict__ tab,
+                                                  bool interleaved) {
+  uint8_t* row0 = tile + r * 128;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const int p = (c ^ (r & 7)) * 16;
+    uint4 x = *reinterpret_cast<uint4*>(row0 + p);               // columns 8c .. 8c+7
+    uint4 y = *reinterpret_cast<uint4*>(row0 + kHalfBytes + p);  // columns 64+8c .. 64+8c+7
+    __nv_bfloat162* xe = reinterpret_cast<__nv_bfloat162*>(&x);
+    __nv_bfloat162* ye = reinterpret_cast<__nv_bfloat162*>(&y);
+    if (!interleaved) {  // pair i = (column i, column i + 64), i = 8c + e
+      const float4* t4 = reinterpret_cast<const float4*>(tab + 8 * c);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 cs = __ldg(t4 + e);  // (cos, sin) of pairs 8c+2e and 8c+2e+1
+        const float2 a = __bfloat1622float2(xe[e]), b = __bfloat1622float2(ye[e]);
+        float a0, b0, a1, b1;
+        rope_rotate(a.x, b.x, cs.x, cs.y, a0, b0);
+        rope_rotate(a.y, b.y, cs.z, cs.w, a1, b1);
+        xe[e] = __floats2bfloat162_rn(a0, a1);
+        ye[e] = __floats2bfloat162_rn(b0, b1);
+      }
+    } else {             // pair i = (column 2i, column 2i + 1): box 0 holds pairs 4c+e, box 1 pairs 32+4c+e
+      const float4* tx = reinterpret_cast<const float4*>(tab + 4 * c);
+      const float4* ty = reinterpret_cast<const float4*>(tab + 32 + 4 * c);
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const float4 cx = __ldg(tx + e), cy = __ldg(ty + e);
+        float2 a = __bfloat1622float2(xe[2 * e]), b = __bfloat1622float2(xe[2 * e + 1]);
+        float r0, r1, r2, r3;
+        rope_rotate(a.x, a.y, cx.x, cx.y, r0, r1);
+        rope_rotate(b.x, b.y, cx.z, cx.w, r2, r3);
+        xe[2 * e] = __floats2bfloat162_rn(r0, r1);
+        xe[2 * e + 1] = __floats2bfloat162_rn(r2, r3);
+        a = __bfloat1622float2(ye[2 * e]);
+        b = __bfloat1622float2(ye[2 * e + 1]);
+        rope_rotate(a.x, a.y, cy.x, cy.y, r0, r1);
+        rope_rotate(b.x, b.y, cy.z, cy.w, r2, r3);
+        ye[2 * e] = __floats2bfloat162_rn(r0, r1);
+        ye[2 * e + 1] = __floats2bfloat162_rn(r2, r3);
+      }
+    }
+    *reinterpret_cast<uint4*>(row0 + p) = x;
+    *reinterpret_cast<uint4*>(row0 + kHalfBytes + p) = y;
+  }
+}
+
+// rope_tab != nullptr: q holds un-rotated queries; each softmax warpgroup rotates its query tile in
+// shared memory once, right after it lands (rope_tab[i * 64 + pair] = (cos, sin) for chunk row i),
+// and the MMA issuer waits for that instead of for the copy.
 __global__ void __launch_bounds__(kAttn2Threads, 1)
 attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ out,
                    float* __restrict__ lse, int Hq, int Hkv, int Lc, int n_cache, float scale_log2,
-                   int32_t* dev_status) {
+                   const float2* __restrict__ rope_tab, int rope_interleaved, int32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
   uint8_t* sQ = smem;                    // [2] query tiles
@@ -126,7 +182,8 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   uint64_t* s_full = bars + 9;    // [2] per tile
   uint64_t* p_ready = bars + 11;  // [2 tiles][2 halves of the key tile]
   uint64_t* o_full = bars + 15;   // [2] per tile
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+  uint64_t* q_rot = bars + 17;    // [2] per tile: query tile rotated in place (rope_tab only)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -150,6 +207,7 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       ptx::mbar_init(p_ready + 2 * s, 128);
       ptx::mbar_init(p_ready + 2 * s + 1, 128);
       ptx::mbar_init(o_full + s, 1);
+      ptx::mbar_init(q_rot + s, 128);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -201,7 +259,9 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     } else if (warp == 9 && lane == 0) {
       const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK), aV = ptx::smem_u32(sV);
       const uint32_t tS0 = tmem_base, tO0 = tmem_base + 128, tS1 = tmem_base + 256, tO1 = tmem_base + 384;
-      bool ok = ptx::mbar_wait(q_full, 0, abort_flag) && ptx::mbar_wait(k_full, 0, abort_flag);
+      bool ok = rope_tab ? ptx::mbar_wait(q_rot, 0, abort_flag) && (!n_kt1 || ptx::mbar_wait(q_rot + 1, 0, abort_flag))
+                         : ptx::mbar_wait(q_full, 0, abort_flag);
+      ok = ok && ptx::mbar_wait(k_full, 0, abort_flag);
       if (ok) {
         ptx::tc_fence_after();
         issue_kmajor_128x128x128(tS0, aQ, aK);
@@ -261,7 +321,13 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int lim = n_cache + row;                // last visible key of this row
     float m = -INFINITY, l0 = 0.f, l1 = 0.f;
     bool ok = tile.n_kt > 0;
-    for (int j = 0; j < tile.n_kt; ++j) {
+    if (rope_tab && ok) {
+      ok = ptx::mbar_wait(q_full, 0, abort_flag);
+      if (ok && row < Lc) rope_rotate_q_row(sQ + t * kTileBytes, r, rope_tab + (long long)row * 64, rope_interleaved != 0);
+      ptx::fence_proxy_async_smem();   // the rotated tile is read by the tensor cores (async proxy)
+      ptx::mbar_arrive(q_rot + t);
+    }
+    for (int j = 0; ok && j < tile.n_kt; ++j) {
       if (!ptx::mbar_wait(s_full + t, j & 1, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
       uint32_t v[128];
@@ -396,7 +462,7 @@ struct ScoreTiles {
 __global__ void __launch_bounds__(kSm100Threads, 2)
 score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                    const float* __restrict__ lse, float* __restrict__ score, int Hq, int Hkv, int Lc,
-                   int n_cache, int cap, int window, float scale_log2, int accumulate,
+                   int n_cache, int cap, int window, float scale_log2, int accumulate, int q_first,
                    int32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
@@ -453,8 +519,9 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         if (!ptx::mbar_wait(q_empty + s, ((it >> 1) & 1) ^ 1, abort_flag)) break;
         ptx::mbar_expect_tx(q_full + s, kTileBytes);
         uint8_t* dst = sQ + s * kTileBytes;
-        ptx::tma_load_3d(dst, &tmQ, q_full + s, 0, t.i0, b * Hq + g * G + t.hh);
-        ptx::tma_load_3d(dst + kHalfBytes, &tmQ, q_full + s, 64, t.i0, b * Hq + g * G + t.hh);
+        // tmQ starts at chunk row q_first (the whole chunk, or a rotated copy of the score window)
+        ptx::tma_load_3d(dst, &tmQ, q_full + s, 0, t.i0 - q_first, b * Hq + g * G + t.hh);
+        ptx::tma_load_3d(dst + kHalfBytes, &tmQ, q_full + s, 64, t.i0 - q_first, b * Hq + g * G + t.hh);
       }
       if (*abort_flag) {
         volatile int ignore = 0;
@@ -535,18 +602,42 @@ inline bool attn_launch_regs_ok() {
   return ok == 1;
 }
 
+// Operands of a step whose rotary embedding is applied inside the call (REFORM_ROPE): the keys
+// rotated at positions 0 .. n-1 into scratch, the queries the score pass reads rotated into
+// scratch, and, for the attention kernel, either rotated queries or the table it rotates with.
+struct RopeOperands {
+  const void* k_rot = nullptr;       // [B*Hkv, cap, 128], the layout of k
+  const void* q_score = nullptr;     // rotated query rows the score pass reads, [B*Hq, q_score_rows, 128]
+  int q_score_rows = 0;              // Lc (all rows) or the score window
+  int q_score_first = 0;             // chunk row of its row 0
+  const void* q_attn = nullptr;      // rotated queries for the attention kernel, or nullptr ...
+  const float2* table = nullptr;     // ... in which case it rotates at load with this table [Lc][64]
+  int interleaved = 0;
+};
+
 // run_attention == false: only the score pass (lse already holds the row normalisers).
 inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float scale, cudaStream_t st,
-                              bool run_attention = true) {
+                              bool run_attention = true, const RopeOperands* rope = nullptr) {
   if (!attn_launch_regs_ok()) return REFORM_ERR_UNSUPPORTED;
   const int n = p->n_cache + p->Lc;
   const float scale_log2 = scale * kLog2e;
-  CUtensorMap tmQ, tmK, tmV;
-  if (!make_tmap_bf16_d128(&tmQ, p->q, (long long)p->B * p->Hq, p->Lc, p->Lc, kT) ||
-      !make_tmap_bf16_d128(&tmK, p->k, (long long)p->B * p->Hkv, n, p->cap, kT) ||
+  CUtensorMap tmQ, tmK, tmV, tmQs;
+  const void* q_attn = rope && rope->q_attn ? rope->q_attn : p->q;
+  const void* k_ptr = rope ? rope->k_rot : p->k;
+  if (!make_tmap_bf16_d128(&tmQ, q_attn, (long long)p->B * p->Hq, p->Lc, p->Lc, kT) ||
+      !make_tmap_bf16_d128(&tmK, k_ptr, (long long)p->B * p->Hkv, n, p->cap, kT) ||
       !make_tmap_bf16_d128(&tmV, p->v, (long long)p->B * p->Hkv, n, p->cap, kT)) {
     g_last_cuda_error = (int)cudaErrorInvalidValue;
     return REFORM_ERR_CUDA;
+  }
+  int q_first = 0;
+  tmQs = tmQ;
+  if (rope && !(p->flags & REFORM_NO_SCORE)) {
+    q_first = rope->q_score_first;
+    if (!make_tmap_bf16_d128(&tmQs, rope->q_score, (long long)p->B * p->Hq, rope->q_score_rows, rope->q_score_rows, kT)) {
+      g_last_cuda_error = (int)cudaErrorInvalidValue;
+      return REFORM_ERR_CUDA;
+    }
   }
   if (run_attention) {
     cudaFuncSetAttribute(attn2_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttn2SmemBytes);
@@ -554,7 +645,7 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
     dim3 grid((units + 1) / 2, p->B * p->Hkv);
     attn2_sm100_kernel<<<grid, kAttn2Threads, kAttn2SmemBytes, st>>>(
         tmQ, tmK, tmV, (__nv_bfloat16*)p->out, lse, p->Hq, p->Hkv, p->Lc, p->n_cache, scale_log2,
-        p->dev_status);
+        rope && !rope->q_attn ? rope->table : nullptr, rope ? rope->interleaved : 0, p->dev_status);
     count_launch();
     int rc = check_launch();
     if (rc != REFORM_OK) return rc;
@@ -563,8 +654,8 @@ inline int launch_chunk_sm100(const reform_chunk_params* p, float* lse, float sc
   cudaFuncSetAttribute(score_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScoreSmemBytes);
   dim3 grid2((n + kT - 1) / kT, p->B * p->Hkv);
   score_sm100_kernel<<<grid2, kSm100Threads, kScoreSmemBytes, st>>>(
-      tmQ, tmK, lse, p->score, p->Hq, p->Hkv, p->Lc, p->n_cache, p->cap, p->score_window, scale_log2,
-      (p->flags & REFORM_SCORE_ACCUMULATE) ? 1 : 0, p->dev_status);
+      tmQs, tmK, lse, p->score, p->Hq, p->Hkv, p->Lc, p->n_cache, p->cap, p->score_window, scale_log2,
+      (p->flags & REFORM_SCORE_ACCUMULATE) ? 1 : 0, q_first, p->dev_status);
   count_launch();
   return check_launch();
 }

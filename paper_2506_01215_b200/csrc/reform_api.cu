@@ -95,6 +95,8 @@ static int validate_chunk(const reform_chunk_params* p) {
     if (!p->score) return REFORM_ERR_INVALID_ARG;
   }
   if (!(p->softmax_scale >= 0.f)) return REFORM_ERR_INVALID_ARG;
+  if ((p->flags & REFORM_ROPE_INTERLEAVED) && !(p->flags & REFORM_ROPE)) return REFORM_ERR_INVALID_ARG;
+  if ((p->flags & REFORM_ROPE) && !(p->rope_theta >= 0.f)) return REFORM_ERR_INVALID_ARG;
   if (!p->q || !p->k || !p->v || !p->out) return REFORM_ERR_INVALID_ARG;
   if (!aligned16(p->q) || !aligned16(p->k) || !aligned16(p->v) || !aligned16(p->out) ||
       !aligned16(p->score) || !aligned16(p->lse))
@@ -104,11 +106,40 @@ static int validate_chunk(const reform_chunk_params* p) {
 }  // namespace reform
 
 namespace reform {
+// Scratch of a REFORM_ROPE step: rotated keys [B*Hkv, cap, d] (the layout of k); rotated queries -- all rows, or on the
+// tensor-core attention path (which rotates its query tiles at load) only the score window's rows;
+// and on that path the (cos, sin) table [Lc][d/2].
+struct RopeScratch {
+  size_t k_bytes, q_bytes, table_bytes;
+  int q_rows, q_first;   // rotated query rows kept, and the chunk row of the first
+  bool at_load;          // the attention kernel rotates its query tiles itself
+  size_t total() const { return k_bytes + q_bytes + table_bytes; }
+};
+
+static RopeScratch rope_scratch(const reform_chunk_params* p) {
+  RopeScratch r{};
+  if (!(p->flags & REFORM_ROPE)) return r;
+  const size_t esz = elem_size(p->dtype);
+  r.at_load = chunk_uses_sm100(p) && !chunk_uses_decode(p);
+  if (r.at_load) {
+    r.q_rows = (p->flags & REFORM_NO_SCORE) ? 0 : p->score_window;
+    r.q_first = p->Lc - r.q_rows;
+    r.table_bytes = align_up(sizeof(float2) * (size_t)p->Lc * (p->d / 2), 256);
+  } else {
+    r.q_rows = p->Lc;
+    r.q_first = 0;
+  }
+  r.k_bytes = align_up((size_t)p->B * p->Hkv * p->cap * p->d * esz, 256);
+  r.q_bytes = align_up((size_t)p->B * p->Hq * r.q_rows * p->d * esz, 256);
+  return r;
+}
+
 static size_t chunk_workspace_bytes(const reform_chunk_params* p) {
   size_t bytes = p->lse ? 0 : chunk_lse_bytes(p);
 #ifndef REFORM_NO_SM100
   if (chunk_uses_decode(p)) bytes += decode_workspace_bytes(p);
 #endif
+  bytes += rope_scratch(p).total();
   return bytes;
 }
 }  // namespace reform
@@ -139,14 +170,76 @@ int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream) {
   float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->d);
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
 #ifndef REFORM_NO_SM100
-  if (chunk_uses_decode(p)) {
-    rc = launch_decode(p, lse, scale, ws, st);
-    if (rc != REFORM_OK || (p->flags & REFORM_NO_SCORE)) return rc;
-    return launch_chunk_sm100(p, lse, scale, st, /*run_attention=*/false);
-  }
-  if (chunk_uses_sm100(p)) return launch_chunk_sm100(p, lse, scale, st);
+  char* ws_decode = ws;
+  if (chunk_uses_decode(p)) ws += decode_workspace_bytes(p);
 #endif
-  return launch_chunk_simt(p, lse, scale, st);
+  if (!(p->flags & REFORM_ROPE)) {
+#ifndef REFORM_NO_SM100
+    if (chunk_uses_decode(p)) {
+      rc = launch_decode(p, lse, scale, ws_decode, st);
+      if (rc != REFORM_OK || (p->flags & REFORM_NO_SCORE)) return rc;
+      return launch_chunk_sm100(p, lse, scale, st, /*run_attention=*/false);
+    }
+    if (chunk_uses_sm100(p)) return launch_chunk_sm100(p, lse, scale, st);
+#endif
+    return launch_chunk_simt(p, lse, scale, st);
+  }
+
+  // REFORM_ROPE: rotate the keys (positions 0 .. n-1) and the queries that are not rotated at load
+  // (positions n_cache + i) into the workspace, then run the same kernels on the rotated operands.
+  const RopeScratch rs = rope_scratch(p);
+  const int n = p->n_cache + p->Lc;
+  const double base = p->rope_theta > 0.f ? (double)p->rope_theta : 10000.0;
+  const bool inter = (p->flags & REFORM_ROPE_INTERLEAVED) != 0;
+  if ((p->d * elem_size(p->dtype)) % 32 != 0) return REFORM_ERR_UNSUPPORTED;
+  void* k_rot = ws;
+  void* q_rot = ws + rs.k_bytes;
+  float2* table = reinterpret_cast<float2*>(ws + rs.k_bytes + rs.q_bytes);
+  if (p->dtype == REFORM_F32) {
+    rc = launch_rope<float>(p->k, k_rot, p->B * p->Hkv, p->d, p->cap, 0, n, 0, base, inter, st);
+    if (rc == REFORM_OK && rs.q_rows)
+      rc = launch_rope<float>(p->q, q_rot, p->B * p->Hq, p->d, p->Lc, rs.q_first, rs.q_rows,
+                              (long long)p->n_cache + rs.q_first, base, inter, st, rs.q_rows, 0);
+  } else {
+    rc = launch_rope<__nv_bfloat16>(p->k, k_rot, p->B * p->Hkv, p->d, p->cap, 0, n, 0, base, inter, st);
+    if (rc == REFORM_OK && rs.q_rows)
+      rc = launch_rope<__nv_bfloat16>(p->q, q_rot, p->B * p->Hq, p->d, p->Lc, rs.q_first, rs.q_rows,
+                                      (long long)p->n_cache + rs.q_first, base, inter, st, rs.q_rows, 0);
+  }
+  if (rc != REFORM_OK) return rc;
+#ifndef REFORM_NO_SM100
+  if (rs.at_load) {
+    rc = launch_rope_table(table, p->Lc, p->d, p->n_cache, base, st);
+    if (rc != REFORM_OK) return rc;
+    RopeOperands ro;
+    ro.k_rot = k_rot;
+    ro.q_score = q_rot;
+    ro.q_score_rows = rs.q_rows;
+    ro.q_score_first = rs.q_first;
+    ro.table = table;
+    ro.interleaved = inter ? 1 : 0;
+    return launch_chunk_sm100(p, lse, scale, st, /*run_attention=*/true, &ro);
+  }
+#endif
+  // every other path reads fully rotated copies: the same kernels on the rotated operands
+  reform_chunk_params r = *p;
+  r.flags &= ~(uint32_t)(REFORM_ROPE | REFORM_ROPE_INTERLEAVED);
+  r.q = q_rot;
+  r.k = k_rot;
+#ifndef REFORM_NO_SM100
+  if (chunk_uses_decode(p)) {
+    rc = launch_decode(&r, lse, scale, ws_decode, st);
+    if (rc != REFORM_OK || (p->flags & REFORM_NO_SCORE)) return rc;
+    RopeOperands ro;
+    ro.k_rot = k_rot;
+    ro.q_score = q_rot;
+    ro.q_score_rows = p->Lc;
+    ro.q_score_first = 0;
+    ro.q_attn = q_rot;
+    return launch_chunk_sm100(p, lse, scale, st, /*run_attention=*/false, &ro);
+  }
+#endif
+  return launch_chunk_simt(&r, lse, scale, st);
 }
 
 /* ---------------------------------------------------------------- evict */
@@ -387,6 +480,7 @@ static int validate_retrieve(const reform_retrieve_params* p) {
     return REFORM_ERR_INVALID_ARG;
   if ((p->E * elem_size(p->dtype)) % 16 != 0) return REFORM_ERR_UNSUPPORTED;
   if (p->pool_window < 1 || p->pool_window % 2 == 0) return REFORM_ERR_INVALID_ARG;
+  if (p->pool_mode != REFORM_POOL_MAX && p->pool_mode != REFORM_POOL_MEAN) return REFORM_ERR_INVALID_ARG;
   if ((p->pool_window - 1) / 2 > kSelMaxRadius) return REFORM_ERR_UNSUPPORTED;
   if (p->k < 0 || p->n_keep_head < 0 || p->n_keep_tail < 0 ||
       (long long)p->n_keep_head + p->n_keep_tail > p->k)
@@ -453,7 +547,7 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
   a.hist = reinterpret_cast<uint32_t*>(ws + L.hist);
   a.blockcnt = reinterpret_cast<uint2*>(ws + L.blockcnt);
   a.blocks_per_seg = L.blocks_per_seg;
-  return launch_select(a, p->B, ts, pooled, (p->pool_window - 1) / 2, ws, L, p->dev_status, st);
+  return launch_select(a, p->B, ts, pooled, (p->pool_window - 1) / 2, ws, L, p->dev_status, st, p->pool_mode);
 }
 
 /* --------------------------------------------------------------- gather */

@@ -20,6 +20,43 @@ struct RopeFreq {
   double turns[kRopeMaxPairs];  // theta_base^(-2 i / d) / (2 pi)
 };
 
+// cos and sin of pos * turns (turns = frequency in turns per position): the product is reduced to
+// [-1/2, 1/2] turns in fp64, and only the reduced angle, as an fp32 value plus its fp32 remainder,
+// goes through the fp32 sincospi.
+__device__ __forceinline__ void rope_cos_sin(double pos, double turns, float& c, float& s) {
+  const double t = pos * turns;
+  const double fr = t - rint(t);           // [-1/2, 1/2] turns, exact
+  const float hi = (float)fr;
+  const float lo = (float)(fr - (double)hi) * 6.2831853071795865f;  // radians left over
+  float sn, cs;
+  sincospif(2.0f * hi, &sn, &cs);
+  c = fmaf(-lo, sn, cs);                   // first-order correction for the remainder
+  s = fmaf(lo, cs, sn);
+}
+
+// Table of (cos, sin) for rows positions pos_begin .. pos_begin + rows - 1 and every pair:
+// tab[r * pairs + i].  Read by the chunk-step kernel that rotates its query tiles at load.
+__global__ void __launch_bounds__(256)
+rope_table_kernel(float2* __restrict__ tab, long long rows, int pairs, long long pos_begin,
+                  const __grid_constant__ RopeFreq freq) {
+  const long long items = rows * pairs;
+  for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < items;
+       it += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(it % pairs);
+    float c, s;
+    rope_cos_sin((double)(pos_begin + it / pairs), freq.turns[i], c, s);
+    tab[it] = make_float2(c, s);
+  }
+}
+
+// The rotation itself, with the roundings spelled out so that every kernel that rotates (this
+// file's and the chunk step's rotation at load) produces the same bits:
+//   a' = fma(a, cos, -(b * sin)),   b' = fma(b, cos, a * sin)
+__device__ __forceinline__ void rope_rotate(float a, float b, float c, float s, float& ra, float& rb) {
+  ra = __fmaf_rn(a, c, -__fmul_rn(b, s));
+  rb = __fmaf_rn(b, c, __fmul_rn(a, s));
+}
+
 // Thread = (row, group of NP consecutive pairs); block = 256 threads.
 //   half layout (interleaved == 0): pair i = (x[i], x[i + d/2]); a thread loads NP consecutive
 //     elements from each half.
@@ -27,7 +64,8 @@ struct RopeFreq {
 template <typename T, bool INTERLEAVED>
 __global__ void __launch_bounds__(256)
 rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long long cap,
-            long long row_begin, long long rows, long long pos_begin, const __grid_constant__ RopeFreq freq) {
+            long long row_begin, long long rows, long long pos_begin, long long dst_cap, long long dst_row_begin,
+            const __grid_constant__ RopeFreq freq) {
   constexpr int NP = 16 / (int)sizeof(T) / (INTERLEAVED ? 2 : 1);  // pairs per thread: one or two 16-byte vectors
   const int groups = (d / 2) / NP;                                  // thread groups per row
   const long long items = rows * groups;
@@ -38,29 +76,22 @@ rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long 
     const double pos = (double)(pos_begin + r);
     float c[NP], s[NP];
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const double t = pos * freq.turns[p0 + i];
-      const double fr = t - rint(t);           // [-1/2, 1/2] turns, exact
-      const float hi = (float)fr;
-      const float lo = (float)(fr - (double)hi) * 6.2831853071795865f;  // radians left over
-      float sn, cs;
-      sincospif(2.0f * hi, &sn, &cs);
-      c[i] = fmaf(-lo, sn, cs);                // first-order correction for the remainder
-      s[i] = fmaf(lo, cs, sn);
-    }
+    for (int i = 0; i < NP; ++i) rope_cos_sin(pos, freq.turns[p0 + i], c[i], s[i]);
 #pragma unroll 4
     for (int bh = 0; bh < BH; ++bh) {
       const long long off = ((long long)bh * cap + row_begin + r) * d;
+      const long long dof = ((long long)bh * dst_cap + dst_row_begin + r) * d;
       if (INTERLEAVED) {
         uint4 v = *reinterpret_cast<const uint4*>(src + off + 2 * p0);
         T* e = reinterpret_cast<T*>(&v);
 #pragma unroll
         for (int i = 0; i < NP; ++i) {
-          const float a = to_float(e[2 * i]), b = to_float(e[2 * i + 1]);
-          e[2 * i] = from_float<T>(a * c[i] - b * s[i]);
-          e[2 * i + 1] = from_float<T>(b * c[i] + a * s[i]);
+          float ra, rb;
+          rope_rotate(to_float(e[2 * i]), to_float(e[2 * i + 1]), c[i], s[i], ra, rb);
+          e[2 * i] = from_float<T>(ra);
+          e[2 * i + 1] = from_float<T>(rb);
         }
-        *reinterpret_cast<uint4*>(dst + off + 2 * p0) = v;
+        *reinterpret_cast<uint4*>(dst + dof + 2 * p0) = v;
       } else {
         uint4 lo = *reinterpret_cast<const uint4*>(src + off + p0);
         uint4 hi = *reinterpret_cast<const uint4*>(src + off + d / 2 + p0);
@@ -68,33 +99,55 @@ rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long 
         T* b = reinterpret_cast<T*>(&hi);
 #pragma unroll
         for (int i = 0; i < NP; ++i) {
-          const float x = to_float(a[i]), y = to_float(b[i]);
-          a[i] = from_float<T>(x * c[i] - y * s[i]);
-          b[i] = from_float<T>(y * c[i] + x * s[i]);
+          float ra, rb;
+          rope_rotate(to_float(a[i]), to_float(b[i]), c[i], s[i], ra, rb);
+          a[i] = from_float<T>(ra);
+          b[i] = from_float<T>(rb);
         }
-        *reinterpret_cast<uint4*>(dst + off + p0) = lo;
-        *reinterpret_cast<uint4*>(dst + off + d / 2 + p0) = hi;
+        *reinterpret_cast<uint4*>(dst + dof + p0) = lo;
+        *reinterpret_cast<uint4*>(dst + dof + d / 2 + p0) = hi;
       }
     }
   }
 }
 
+inline RopeFreq rope_freq(int d, double base) {
+  RopeFreq freq;
+  for (int i = 0; i < d / 2; ++i) freq.turns[i] = pow(base, -2.0 * i / d) / 6.283185307179586476925;
+  return freq;
+}
+
+inline int launch_rope_table(float2* tab, long long rows, int d, long long pos_begin, double base, cudaStream_t st) {
+  if (rows == 0) return REFORM_OK;
+  const long long items = rows * (d / 2);
+  long long blocks = (items + 255) / 256;
+  const long long cap_blocks = (long long)num_sms() * 16;
+  rope_table_kernel<<<(int)(blocks < cap_blocks ? blocks : cap_blocks), 256, 0, st>>>(tab, rows, d / 2, pos_begin,
+                                                                                       rope_freq(d, base));
+  count_launch();
+  return check_launch();
+}
+
+// dst_cap / dst_row_begin: row capacity per (batch, head) of dst and the row of dst that receives
+// the first rotated row (negative dst_cap: same layout as src).
 template <typename T>
 inline int launch_rope(const void* src, void* dst, int BH, int d, long long cap, long long row_begin,
                        long long rows, long long pos_begin, double base, bool interleaved,
-                       cudaStream_t st) {
+                       cudaStream_t st, long long dst_cap = -1, long long dst_row_begin = 0) {
   if (rows == 0 || BH == 0) return REFORM_OK;
+  if (dst_cap < 0) { dst_cap = cap; dst_row_begin = row_begin; }
   const int np = 16 / (int)sizeof(T) / (interleaved ? 2 : 1);
   const long long items = rows * ((d / 2) / np);
   long long blocks = (items + 255) / 256;
   const long long cap_blocks = (long long)num_sms() * 16;
   const int grid = (int)(blocks < cap_blocks ? blocks : cap_blocks);
-  RopeFreq freq;
-  for (int i = 0; i < d / 2; ++i) freq.turns[i] = pow(base, -2.0 * i / d) / 6.283185307179586476925;
+  const RopeFreq freq = rope_freq(d, base);
   if (interleaved)
-    rope_kernel<T, true><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, freq);
+    rope_kernel<T, true><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin,
+                                               dst_cap, dst_row_begin, freq);
   else
-    rope_kernel<T, false><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin, freq);
+    rope_kernel<T, false><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin,
+                                                dst_cap, dst_row_begin, freq);
   count_launch();
   return check_launch();
 }

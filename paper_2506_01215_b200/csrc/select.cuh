@@ -158,13 +158,71 @@ __device__ __forceinline__ void sel_pass_params(int pass, int& shift, uint32_t& 
   else { shift = 0; digit_mask = 0x3FFu; prefix_mask = 0xFFFFFC00u; }
 }
 
+// Pools the raw token scores of one block's tile (Sec. 3.3).  tile: 2 * (kSelTile + 2 * radius)
+// floats of shared memory.  On return pooled_of(i) for the block's element i (0 <= i < kSelTile)
+// is available through pool_result().  mode 0: maximum over the clipped window by log-step
+// doubling; mode 1: mean over the clipped window by direct summation in ascending token order.
+struct PoolTile {
+  float* cur;      // after pool_prepare: the array pool_result reads
+  int radius, window, len, mode;
+  long long base;  // first token of the block's tile
+  int n;
+};
+
+__device__ __forceinline__ PoolTile pool_prepare(float* tile, const float* __restrict__ src, long long base, int n,
+                                                 int radius, int mode) {
+  const int tid = threadIdx.x;
+  const int span = kSelTile + 2 * radius;
+  PoolTile p;
+  p.radius = radius;
+  p.window = 2 * radius + 1;
+  p.mode = mode;
+  p.base = base;
+  p.n = n;
+  float* cur = tile;
+  float* nxt = tile + span;
+  for (int i = tid; i < span; i += kSelThreads) {
+    long long g = base - radius + i;
+    cur[i] = (g >= 0 && g < n) ? src[g] : -INFINITY;
+  }
+  __syncthreads();
+  int len = 1;
+  if (mode == 0) {
+    // W_p[j] = max cur[j .. j + 2^p - 1], doubling p while 2^(p+1) <= window
+    while (2 * len <= p.window) {
+      for (int i = tid; i < span; i += kSelThreads) {
+        float v = cur[i];
+        if (i + len < span) v = fmaxf(v, cur[i + len]);
+        nxt[i] = v;
+      }
+      __syncthreads();
+      float* t = cur; cur = nxt; nxt = t;
+      len *= 2;
+    }
+  }
+  p.cur = cur;
+  p.len = len;
+  return p;
+}
+
+// pooled score of the tile's element i (token base + i, which must be < n)
+__device__ __forceinline__ float pool_result(const PoolTile& p, int i) {
+  if (p.mode == 0) return fmaxf(p.cur[i], p.cur[i + p.window - p.len]);  // max(W[c], W[c + window - len])
+  const long long g = p.base + i;
+  const int lo = (int)(g - p.radius < 0 ? -g : -p.radius);                  // offsets of the clipped window
+  const int hi = (int)(g + p.radius > p.n - 1 ? p.n - 1 - g : p.radius);
+  float sum = 0.f;
+  for (int u = lo; u <= hi; ++u) sum += p.cur[i + p.radius + u];
+  return sum / (float)(hi - lo + 1);
+}
+
 // One histogram pass.  POOL (pass 0 only): vals_in holds the raw token scores
 // ts; the block computes pooled[i] = max ts[i-r .. i+r] (clipped), writes it
 // to pooled_out, and histograms that.
 template <bool POOL>
 __global__ void __launch_bounds__(kSelThreads)
 sel_hist_kernel(SelArgs a, int pass, const float* __restrict__ ts, float* __restrict__ pooled_out,
-                int radius) {
+                int radius, int pool_mode) {
   extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
   __shared__ uint32_t hist[kSelBins];
   __shared__ uint32_t scratch[33];
@@ -180,34 +238,12 @@ sel_hist_kernel(SelArgs a, int pass, const float* __restrict__ ts, float* __rest
   const long long base = (long long)blockIdx.x * kSelTile;  // offset inside [0, n)
   if (POOL) {
     // tile covers ts[base - radius, base + kSelTile + radius)
-    const int span = kSelTile + 2 * radius;
-    float* cur = tile;
-    float* nxt = tile + span;
-    const float* src = ts + (long long)seg * a.stride;
-    for (int i = tid; i < span; i += kSelThreads) {
-      long long g = base - radius + i;
-      cur[i] = (g >= 0 && g < a.n) ? src[g] : -INFINITY;
-    }
-    __syncthreads();
-    // W_p[j] = max cur[j .. j + 2^p - 1], doubling p while 2^(p+1) <= window
-    const int window = 2 * radius + 1;
-    int len = 1;
-    while (2 * len <= window) {
-      for (int i = tid; i < span; i += kSelThreads) {
-        float v = cur[i];
-        if (i + len < span) v = fmaxf(v, cur[i + len]);
-        nxt[i] = v;
-      }
-      __syncthreads();
-      float* t = cur; cur = nxt; nxt = t;
-      len *= 2;
-    }
-    // window max at centre c (tile index c + radius) = max(W[c], W[c + window - len])
+    const PoolTile pt = pool_prepare(tile, ts + (long long)seg * a.stride, base, a.n, radius, pool_mode);
     float* dst = pooled_out + (long long)seg * a.stride;
     for (int j = 0; j < kSelPerThread; ++j) {
       int i = j * kSelThreads + tid;
       long long g = base + i;
-      const float v = fmaxf(cur[i], cur[i + window - len]);
+      const float v = g < a.n ? pool_result(pt, i) : 0.f;
       if (g < a.n) dst[g] = v;
       hist_add(hist, float_to_key(v) >> shift, g >= a.lo && g < a.hi);  // every lane calls; hi <= n
     }
@@ -390,7 +426,7 @@ __device__ __forceinline__ void sel_find_bin_local(const uint32_t* hist, uint32_
 template <bool POOL>
 __global__ void __launch_bounds__(kSelThreads)
 sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
-                 float* __restrict__ pooled_out, int radius, int32_t* dev_status) {
+                 float* __restrict__ pooled_out, int radius, int pool_mode, int32_t* dev_status) {
   extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
   __shared__ uint32_t hist[kSelBins];
   __shared__ uint32_t scratch[33];
@@ -403,27 +439,7 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
   bool cand[kSelPerThread];
 
   if (POOL) {
-    const int span = kSelTile + 2 * radius;
-    float* cur = tile;
-    float* nxt = tile + span;
-    const float* src = ts + (long long)seg * a.stride;
-    for (int i = tid; i < span; i += kSelThreads) {
-      long long g = base - radius + i;
-      cur[i] = (g >= 0 && g < a.n) ? src[g] : -INFINITY;
-    }
-    __syncthreads();
-    const int window = 2 * radius + 1;
-    int len = 1;
-    while (2 * len <= window) {
-      for (int i = tid; i < span; i += kSelThreads) {
-        float v = cur[i];
-        if (i + len < span) v = fmaxf(v, cur[i + len]);
-        nxt[i] = v;
-      }
-      __syncthreads();
-      float* t = cur; cur = nxt; nxt = t;
-      len *= 2;
-    }
+    const PoolTile pt = pool_prepare(tile, ts + (long long)seg * a.stride, base, a.n, radius, pool_mode);
     float* dst = pooled_out + (long long)seg * a.stride;
 #pragma unroll
     for (int j = 0; j < kSelPerThread; ++j) {
@@ -432,7 +448,7 @@ sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
       cand[j] = g >= a.lo && g < a.hi;
       key[j] = 0;
       if (g < a.n) {
-        float v = fmaxf(cur[i], cur[i + window - len]);
+        float v = pool_result(pt, i);
         dst[g] = v;
         key[j] = float_to_key(v);
       }
@@ -647,7 +663,8 @@ inline int sel_fused_capacity(size_t smem) {
 }
 
 inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, int radius,
-                         void* ws_base, const SelLayout& L, int32_t* dev_status, cudaStream_t st) {
+                         void* ws_base, const SelLayout& L, int32_t* dev_status, cudaStream_t st,
+                         int pool_mode = 0) {
   if (segs == 0) return REFORM_OK;
   if (!ts && a.n <= kSelBlockMaxN && segs >= kSelBlockMinSegs) {
     sel_block_kernel<<<segs, kSelThreads, 0, st>>>(a);
@@ -662,7 +679,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
     if ((long long)a.blocks_per_seg * segs <= capacity) {
       if (cudaMemsetAsync(ws_base, 0, L.zero_bytes, st) != cudaSuccess) return check_launch();
       SelFusedCtl* ctl = reinterpret_cast<SelFusedCtl*>(reinterpret_cast<char*>(ws_base) + L.ctl);
-      void* args[] = {&a, &ctl, &ts, &pooled, &radius, &dev_status};
+      void* args[] = {&a, &ctl, &ts, &pooled, &radius, &pool_mode, &dev_status};
       cudaError_t e = cudaLaunchCooperativeKernel(
           ts ? (const void*)sel_fused_kernel<true> : (const void*)sel_fused_kernel<false>, grid,
           dim3(kSelThreads), args, smem, st);
@@ -679,12 +696,12 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
   if (ts) {
     size_t smem = sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius);
     cudaFuncSetAttribute(sel_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    sel_hist_kernel<true><<<grid, kSelThreads, smem, st>>>(a, 0, ts, pooled, radius);
+    sel_hist_kernel<true><<<grid, kSelThreads, smem, st>>>(a, 0, ts, pooled, radius, pool_mode);
   } else {
-    sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 0, nullptr, nullptr, 0);
+    sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 0, nullptr, nullptr, 0, 0);
   }
-  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 1, nullptr, nullptr, 0);
-  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 2, nullptr, nullptr, 0);
+  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 1, nullptr, nullptr, 0, 0);
+  sel_hist_kernel<false><<<grid, kSelThreads, 0, st>>>(a, 2, nullptr, nullptr, 0, 0);
   sel_count_kernel<<<grid, kSelThreads, 0, st>>>(a);
   sel_write_kernel<<<grid, kSelThreads, 0, st>>>(a);
   count_launch(5);

@@ -410,6 +410,30 @@ def test_retrieve_matches_oracle(name, N, pool, keep, k):
             assert set(planted[b]) <= set(idx[b].tolist())
 
 
+@pytest.mark.parametrize("name,N,pool,keep,k", [
+    ("tiny", 8192, 21, 8, 256),                # fp32, the paper's 20 neighbours
+    ("tiny", 5000, 5, 0, 300),
+    ("llama8b_128k", 9001, 21, 256, 1024),     # bf16 tensor-core scan, ragged, several selection blocks
+    ("mistral7b_4x256k", 3000, 129, 16, 700),  # batch 4, a window of 129
+])
+def test_retrieve_with_mean_pooling_matches_oracle(name, N, pool, keep, k):
+    """The mean-pool scorer variant (Appendix, detailed head selection, Step 3) through the same call."""
+    w = dataclasses.replace(synth.WORKLOADS[name], N=N, k=k, pool_window=pool, keep_head=keep, keep_tail=keep)
+    bank, qs, planted = synth.bank_and_queries(w, seed=N + pool)
+    p = dict(scale=w.sim_scale, pool_window=pool, n_keep_head=keep, n_keep_tail=keep)
+    ref = oracle.retrieve_topk(bank, qs, N, k, pool_mode="mean", **p)
+    idx = torch.full((w.B, k), -1, dtype=torch.int32, device=DEV)
+    ts = torch.zeros(w.B, N, device=DEV)
+    pooled = torch.zeros(w.B, N, device=DEV)
+    R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx, token_score_out=ts, pooled_score_out=pooled,
+                    pool_mode=R.POOL_MEAN, **p)
+    torch.cuda.synchronize()
+    assert_scores_close(ts, ref["ts"], 1.0)
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    for b in range(w.B):
+        assert_index_sets_match(idx[b].cpu(), ref["idx"][b], ref["pooled"][b])
+
+
 def test_retrieve_window_wider_than_the_bank():
     g = torch.Generator().manual_seed(12)
     bank = torch.randn(2, 50, 64, generator=g).bfloat16()
@@ -654,3 +678,51 @@ def test_chunk_step_on_rotated_operands():
     assert_outputs_close(out, o_ref, torch.bfloat16)
     s_ref = oracle.key_scores(qo, ko, n_cache, 128, score_in=carry, accumulate=True)
     assert_scores_close(score[:, :, :n], s_ref[:, :, :n], 128 * 4 / n)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,d,Lc,n_cache,dtype,W,flags,theta", [
+    (1, 8, 2, 128, 300, 200, torch.bfloat16, 128, 0, 0.0),                 # tensor-core path: query tiles rotated at load
+    (2, 4, 2, 128, 257, 0, torch.bfloat16, 257, 0, 500000.0),              # first step, every row scores, Llama-3 base
+    (1, 8, 2, 128, 200, 5000, torch.bfloat16, 64, R.ROPE_INTERLEAVED, 0.0),  # interleaved pairs, positions in the thousands
+    (1, 4, 1, 128, 129, 77, torch.bfloat16, 1, R.NO_SCORE, 0.0),           # attention only
+    (1, 4, 2, 64, 192, 100, torch.float32, 128, 0, 0.0),                   # CUDA-core path (Tiny's shapes)
+    (1, 8, 2, 128, 1, 1500, torch.bfloat16, 1, 0, 0.0),                    # decode-shaped step
+    (1, 4, 2, 64, 96, 40, torch.bfloat16, 32, R.ROPE_INTERLEAVED, 0.0),    # bf16 on the CUDA-core path
+])
+def test_chunk_step_applies_rope_inside_the_call(B, Hq, Hkv, d, Lc, n_cache, dtype, W, flags, theta):
+    """REFORM_ROPE: the caller passes un-rotated queries and keys (the cache keeps them un-rotated,
+    because every compression renumbers its rows) and the call rotates them at the ids of the moment
+    -- cache and chunk keys at 0 .. n-1, chunk queries at n_cache + i -- before attending and
+    scoring; q and k are left as they were.  Against the oracle rotating in fp64 and then attending."""
+    q, k, v, carry = _case(B, Hq, Hkv, d, Lc, n_cache, dtype, seed=Lc + n_cache)
+    n = n_cache + Lc
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    out = torch.full_like(qd, float("nan"))
+    lse = torch.full(q.shape[:3], float("nan"), device=DEV)
+    score = carry.to(DEV).clone()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.chunk_step(qd, kd, vd, out, score, n_cache, W, lse=lse, flags=R.SCORE_ACCUMULATE | R.ROPE | flags,
+                 rope_theta=theta, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(qd.cpu(), q) and torch.equal(kd.cpu(), k)          # inputs untouched
+    base = theta or 10000.0
+    inter = bool(flags & R.ROPE_INTERLEAVED)
+    qo = oracle.rope(q, 0, Lc, n_cache, base=base, interleaved=inter)
+    ko = oracle.rope(k, 0, n, 0, base=base, interleaved=inter)
+    o_ref, l_ref = oracle.attention(qo, ko, v, n_cache)
+    assert_outputs_close(out, o_ref, dtype)
+    assert (lse.cpu().double() - l_ref).abs().max() < (3e-3 if dtype == torch.bfloat16 else 1e-4)
+    if flags & R.NO_SCORE:
+        assert torch.equal(score.cpu(), carry)
+    else:
+        s_ref = oracle.key_scores(qo, ko, n_cache, W, score_in=carry, accumulate=True)
+        assert_scores_close(score[:, :, :n], s_ref[:, :, :n], W * (Hq // Hkv) / n)
+    # and it equals the two-call form (reform_rope, then the plain step) bit for bit
+    q_rot, k_rot = torch.empty_like(qd), kd.clone()
+    R.rope(qd, q_rot, 0, Lc, n_cache, theta_base=theta, interleaved=inter)
+    R.rope(kd, k_rot, 0, n, 0, theta_base=theta, interleaved=inter)
+    out2 = torch.empty_like(qd)
+    score2 = carry.to(DEV).clone()
+    R.chunk_step(q_rot, k_rot, vd, out2, score2, n_cache, W, flags=R.SCORE_ACCUMULATE | (flags & R.NO_SCORE))
+    assert torch.equal(out2, out) and torch.equal(score2, score)

@@ -98,6 +98,7 @@ def test_struct_layouts_match_the_header():
 @pytest.mark.parametrize("kw", [
     dict(Hq=5), dict(n_cache=8), dict(score_window=0), dict(score_window=65), dict(q=None),
     dict(score=None), dict(q=FAKE + 4), dict(softmax_scale=-1.0), dict(struct_size=0),
+    dict(flags=R.ROPE_INTERLEAVED), dict(flags=R.ROPE, rope_theta=-2.0),
 ])
 def test_chunk_step_rejects_bad_arguments(kw):
     assert R.lib().reform_chunk_step(ctypes.byref(_chunk(**kw)), None) == R.ERR_INVALID_ARG
@@ -146,7 +147,7 @@ def test_evict_reports_n_kept_and_needs_workspace():
 
 @pytest.mark.parametrize("kw", [
     dict(pool_window=4), dict(pool_window=0), dict(n_keep_head=10, n_keep_tail=10), dict(N=2000),
-    dict(nq=0), dict(bank=None), dict(idx_out=FAKE + 8),
+    dict(nq=0), dict(bank=None), dict(idx_out=FAKE + 8), dict(pool_mode=2), dict(pool_mode=-1),
 ])
 def test_retrieve_rejects_bad_arguments(kw):
     assert R.lib().reform_retrieve_topk(ctypes.byref(_retrieve(**kw)), None) == R.ERR_INVALID_ARG

@@ -353,6 +353,39 @@ def test_retrieve_matches_library_matmul_pool_and_sort(pool):
         assert r["idx"][b].tolist() == expect
 
 
+@pytest.mark.parametrize("pool", [1, 5, 21, 601])
+def test_retrieve_mean_pooling_matches_library_avg_pool(pool):
+    """The mean-pool smoothing of the head-ranking procedure (Appendix, detailed head selection,
+    Step 3): mean over the token and its neighbours, over the tokens that exist at the ends ==
+    library avg_pool1d without counting the padding; selection by a stable sort of that."""
+    g = torch.Generator().manual_seed(13)
+    B, N, E, nq, k = 2, 300, 24, 3, 40
+    bank = torch.randn(B, N + 5, E, generator=g).bfloat16()
+    qs = torch.randn(B, nq, E, generator=g).bfloat16()
+    r = oracle.retrieve_topk(bank, qs, N, k, scale=0.5, pool_window=pool, n_keep_head=4, n_keep_tail=6,
+                             pool_mode="mean")
+    ts = (0.5 * (qs.double() @ bank[:, :N].double().transpose(1, 2))).max(dim=1).values
+    assert torch.allclose(r["ts"], ts, atol=1e-13)
+    if pool // 2 < N:
+        pooled = torch.nn.functional.avg_pool1d(ts[:, None], kernel_size=pool, stride=1, padding=pool // 2,
+                                                count_include_pad=False)[:, 0]
+    else:                                       # window wider than the bank: the mean of everything
+        pooled = ts.mean(dim=1, keepdim=True).expand(B, N)
+    assert torch.allclose(r["pooled"], pooled, atol=1e-12)
+    # brute force at a few tokens, both ends included
+    rad = pool // 2
+    for t in (0, 1, min(rad, N - 1), N // 2, N - 2, N - 1):
+        lo, hi = max(0, t - rad), min(N - 1, t + rad)
+        assert abs(float(r["pooled"][1, t]) - float(ts[1, lo:hi + 1].sum() / (hi - lo + 1))) < 1e-12
+    for b in range(B):
+        mid = r["pooled"][b, 4:N - 6]
+        order = torch.sort(mid, descending=True, stable=True).indices[:k - 10] + 4
+        assert r["idx"][b].tolist() == sorted(list(range(4)) + order.tolist() + list(range(N - 6, N)))
+    # a constant stays constant, and the mean never exceeds the max-pooled score
+    rmax = oracle.retrieve_topk(bank, qs, N, k, scale=0.5, pool_window=pool, n_keep_head=4, n_keep_tail=6)
+    assert (r["pooled"] <= rmax["pooled"] + 1e-15).all()
+
+
 def test_retrieve_self_similarity_orthogonality_and_bound():
     E = 16
     eye = torch.eye(E)
