@@ -30,6 +30,9 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--simt", action="store_true")
     ap.add_argument("--no-score", action="store_true", help="chunk_step without the key-score pass")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the call in a CUDA graph and time its replays (device time without the "
+                         "host's launch cost)")
     a = ap.parse_args()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
@@ -79,12 +82,26 @@ def main():
         fn = lambda: R.gather(hidden, idx, dst)
     fn()
     torch.cuda.synchronize()
+    run = fn
+    if a.graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            fn()
+        run = graph.replay
+        run()
+        torch.cuda.synchronize()
     ev0.record()
     for _ in range(a.reps):
-        fn()
+        run()
     ev1.record()
     torch.cuda.synchronize()
-    print(f"{a.op}: {ev0.elapsed_time(ev1) / a.reps:.4f} ms per call over {a.reps} calls")
+    how = "graph replays" if a.graph else "calls"
+    print(f"{a.op}: {ev0.elapsed_time(ev1) / a.reps:.4f} ms per call over {a.reps} {how}")
 
 
 if __name__ == "__main__":
