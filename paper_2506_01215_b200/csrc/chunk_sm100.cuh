@@ -112,9 +112,9 @@ __device__ __forceinline__ Attn2Tile attn2_tile(int u, int U, int G, int n_qt, i
 // position n_cache + i once the cache rows have been renumbered).  The tile is two boxes of 64
 // columns, 128 bytes per row, 16-byte chunks XOR-swizzled by (row & 7); column c of box 0 and
 // column c of box 1 share an offset, which is where the two halves of a rotate-half pair live.
-// tab: the row's 64 (cos, sin) pairs.
-__device__ __forceinline__ void rope_rotate_q_row(uint8_t* tile, int r, const float2* __restrict__ tab,
-                                                  bool interleaved) {
+// tab: the row's 64 (cos, sin) pairs as 32 float4, fetched by the caller before it waited for the
+// tile (the table does not depend on the tile, so its latency hides under the tile's copy).
+__device__ __forceinline__ void rope_rotate_q_row(uint8_t* tile, int r, const float4 (&tab)[32], bool interleaved) {
   uint8_t* row0 = tile + r * 128;
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
@@ -124,10 +124,9 @@ __device__ __forceinline__ void rope_rotate_q_row(uint8_t* tile, int r, const fl
     __nv_bfloat162* xe = reinterpret_cast<__nv_bfloat162*>(&x);
     __nv_bfloat162* ye = reinterpret_cast<__nv_bfloat162*>(&y);
     if (!interleaved) {  // pair i = (column i, column i + 64), i = 8c + e
-      const float4* t4 = reinterpret_cast<const float4*>(tab + 8 * c);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float4 cs = __ldg(t4 + e);  // (cos, sin) of pairs 8c+2e and 8c+2e+1
+        const float4 cs = tab[4 * c + e];  // (cos, sin) of pairs 8c+2e and 8c+2e+1
         const float2 a = __bfloat1622float2(xe[e]), b = __bfloat1622float2(ye[e]);
         float a0, b0, a1, b1;
         rope_rotate(a.x, b.x, cs.x, cs.y, a0, b0);
@@ -136,11 +135,9 @@ __device__ __forceinline__ void rope_rotate_q_row(uint8_t* tile, int r, const fl
         ye[e] = __floats2bfloat162_rn(b0, b1);
       }
     } else {             // pair i = (column 2i, column 2i + 1): box 0 holds pairs 4c+e, box 1 pairs 32+4c+e
-      const float4* tx = reinterpret_cast<const float4*>(tab + 4 * c);
-      const float4* ty = reinterpret_cast<const float4*>(tab + 32 + 4 * c);
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        const float4 cx = __ldg(tx + e), cy = __ldg(ty + e);
+        const float4 cx = tab[2 * c + e], cy = tab[16 + 2 * c + e];
         float2 a = __bfloat1622float2(xe[2 * e]), b = __bfloat1622float2(xe[2 * e + 1]);
         float r0, r1, r2, r3;
         rope_rotate(a.x, a.y, cx.x, cx.y, r0, r1);
@@ -322,8 +319,12 @@ attn2_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     float m = -INFINITY, l0 = 0.f, l1 = 0.f;
     bool ok = tile.n_kt > 0;
     if (rope_tab && ok) {
+      float4 tab[32];   // this row's 64 (cos, sin) pairs, on their way while the tile's copy is in flight
+      const float4* tr = reinterpret_cast<const float4*>(rope_tab + (long long)min(row, Lc - 1) * 64);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) tab[i] = __ldg(tr + i);
       ok = ptx::mbar_wait(q_full, 0, abort_flag);
-      if (ok && row < Lc) rope_rotate_q_row(sQ + t * kTileBytes, r, rope_tab + (long long)row * 64, rope_interleaved != 0);
+      if (ok && row < Lc) rope_rotate_q_row(sQ + t * kTileBytes, r, tab, rope_interleaved != 0);
       ptx::fence_proxy_async_smem();   // the rotated tile is read by the tensor cores (async proxy)
       ptx::mbar_arrive(q_rot + t);
     }
@@ -591,13 +592,15 @@ score_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   if (threadIdx.x == 0 && *abort_flag) report_device_error(dev_status, REFORM_DEV_TIMEOUT);
 }
 
-// The setmaxnreg split above assumes the register count the compiler gave the kernel at launch;
-// refuse to launch if it ever differs (an unsatisfiable increase would block forever).
+// The setmaxnreg split above draws on the registers the block is launched with: 384 threads times
+// the kernel's register count.  If a compiler ever gave the kernel fewer than the split needs, the
+// increase could not be met and would block forever, so such a build refuses to launch (with 384
+// threads per block the count cannot exceed 168, and any count from 168 up holds the split).
 inline bool attn_launch_regs_ok() {
   static int ok = -1;
   if (ok < 0) {
     cudaFuncAttributes a2;
-    ok = cudaFuncGetAttributes(&a2, attn2_sm100_kernel) == cudaSuccess && a2.numRegs == kAttn2LaunchRegs;
+    ok = cudaFuncGetAttributes(&a2, attn2_sm100_kernel) == cudaSuccess && a2.numRegs >= kAttn2LaunchRegs;
   }
   return ok == 1;
 }

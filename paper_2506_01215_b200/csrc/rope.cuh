@@ -77,8 +77,11 @@ rope_kernel(const T* __restrict__ src, T* __restrict__ dst, int BH, int d, long 
     float c[NP], s[NP];
 #pragma unroll
     for (int i = 0; i < NP; ++i) rope_cos_sin(pos, freq.turns[p0 + i], c[i], s[i]);
+    // blockIdx.y splits the (batch, head) range when there are too few rows to fill the device
+    const int bh_per = (BH + (int)gridDim.y - 1) / (int)gridDim.y;
+    const int bh_begin = (int)blockIdx.y * bh_per, bh_end = min(BH, bh_begin + bh_per);
 #pragma unroll 4
-    for (int bh = 0; bh < BH; ++bh) {
+    for (int bh = bh_begin; bh < bh_end; ++bh) {
       const long long off = ((long long)bh * cap + row_begin + r) * d;
       const long long dof = ((long long)bh * dst_cap + dst_row_begin + r) * d;
       if (INTERLEAVED) {
@@ -140,7 +143,12 @@ inline int launch_rope(const void* src, void* dst, int BH, int d, long long cap,
   const long long items = rows * ((d / 2) / np);
   long long blocks = (items + 255) / 256;
   const long long cap_blocks = (long long)num_sms() * 16;
-  const int grid = (int)(blocks < cap_blocks ? blocks : cap_blocks);
+  const int grid_x = (int)(blocks < cap_blocks ? blocks : cap_blocks);
+  // few rows (a score window, a decode step): spread the (batch, head) loop over blockIdx.y as well
+  int grid_y = 1;
+  while (grid_x * grid_y < 2 * num_sms() && grid_y < BH) grid_y *= 2;
+  if (grid_y > BH) grid_y = BH;
+  const dim3 grid(grid_x, grid_y);
   const RopeFreq freq = rope_freq(d, base);
   if (interleaved)
     rope_kernel<T, true><<<grid, 256, 0, st>>>((const T*)src, (T*)dst, BH, d, cap, row_begin, rows, pos_begin,

@@ -30,6 +30,7 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--simt", action="store_true")
     ap.add_argument("--no-score", action="store_true", help="chunk_step without the key-score pass")
+    ap.add_argument("--rope", action="store_true", help="chunk_step on un-rotated operands (REFORM_ROPE)")
     ap.add_argument("--graph", action="store_true",
                     help="capture the call in a CUDA graph and time its replays (device time without the "
                          "host's launch cost)")
@@ -50,7 +51,8 @@ def main():
     if a.op == "chunk_step":
         out = torch.empty_like(q)
         lse = torch.empty(q.shape[:3], dtype=torch.float32, device=dev)
-        flags = (R.NO_SCORE if a.no_score else R.SCORE_ACCUMULATE) | (R.FORCE_SIMT if a.simt else 0)
+        flags = (R.NO_SCORE if a.no_score else R.SCORE_ACCUMULATE) | (R.FORCE_SIMT if a.simt else 0) | \
+            (R.ROPE if a.rope else 0)
         fn = lambda: R.chunk_step(q, k, v, out, score, w.budget, w.window, lse=lse, flags=flags)
     elif a.op == "evict":
         kd, vd, sd = torch.empty_like(k), torch.empty_like(v), torch.empty_like(score)

@@ -726,3 +726,62 @@ def test_chunk_step_applies_rope_inside_the_call(B, Hq, Hkv, d, Lc, n_cache, dty
     score2 = carry.to(DEV).clone()
     R.chunk_step(q_rot, k_rot, vd, out2, score2, n_cache, W, flags=R.SCORE_ACCUMULATE | (flags & R.NO_SCORE))
     assert torch.equal(out2, out) and torch.equal(score2, score)
+
+
+def test_checkpoint_and_resume_is_bit_identical():
+    """All recurrent state is caller-owned (cache K/V, carried scores, n_cache, bank rows written so
+    far), so a checkpoint is a copy of those buffers: 8 chunk steps straight against 4 steps,
+    copy-out to the host, copy-in to fresh buffers, 4 more steps -- the same bits everywhere."""
+    w = synth.WORKLOADS["tiny"]
+    sel = synth.head_selection(dataclasses.replace(w, n_slots=2, slot_dim=w.d))
+    E = 2 * w.d
+
+    def new_state():
+        cache = LayerCache(w.B, w.Hkv, w.d, w.cap, w.budget, w.n_sink, w.n_recent, w.dtype, DEV)
+        bank = torch.zeros(w.B, w.T, E, dtype=w.dtype, device=DEV)
+        return cache, bank
+
+    def run(cache, bank, steps):
+        out = torch.zeros(w.B, w.Hq, w.Lc, w.d, device=DEV)
+        outs = []
+        for step in steps:
+            q, kc, vc = synth.chunk_qkv(w, 0, step)
+            q, kc, vc = q.to(DEV), kc.to(DEV), vc.to(DEV)
+            cache.write_chunk(kc, vc)
+            cache.attend(q, out, w.window)
+            R.embed_append(bank, step * w.Lc, sel, q_state=q, k_state=kc, v_state=vc)
+            cache.evict()
+            outs.append(out.clone())
+        return outs
+
+    c1, b1 = new_state()
+    outs1 = run(c1, b1, range(8))
+    c2, b2 = new_state()
+    outs2 = run(c2, b2, range(4))
+    # checkpoint: everything the recurrence carries, to the host ...
+    ck = dict(k=c2.k[c2.cur].cpu(), v=c2.v[c2.cur].cpu(), score=c2.score[c2.cur].cpu(), n_cache=c2.n_cache,
+              bank=b2.cpu())
+    del c2, b2
+    # ... and back into fresh buffers
+    c3, b3 = new_state()
+    c3.k[c3.cur].copy_(ck["k"])
+    c3.v[c3.cur].copy_(ck["v"])
+    c3.score[c3.cur].copy_(ck["score"])
+    c3.n_cache = c3.n_keys = ck["n_cache"]
+    b3.copy_(ck["bank"])
+    outs2 += run(c3, b3, range(4, 8))
+    for a, b in zip(outs1, outs2):
+        assert torch.equal(a, b)
+    n = c1.n_cache
+    assert c3.n_cache == n == w.budget
+    assert torch.equal(c1.k[c1.cur][:, :, :n], c3.k[c3.cur][:, :, :n])
+    assert torch.equal(c1.v[c1.cur][:, :, :n], c3.v[c3.cur][:, :, :n])
+    assert torch.equal(c1.score[c1.cur][:, :, :n], c3.score[c3.cur][:, :, :n])
+    assert torch.equal(b1, b3)
+    # and the gather phase over the resumed bank picks the same tokens
+    _, queries, _ = synth.bank_and_queries(dataclasses.replace(w, n_slots=2, slot_dim=w.d, N=256, n_planted=0))
+    idx = [torch.zeros(w.B, w.k, dtype=torch.int32, device=DEV) for _ in range(2)]
+    for bank, i in ((b1, idx[0]), (b3, idx[1])):
+        R.retrieve_topk(bank, queries.to(DEV), w.T, w.k, i, scale=0.5, pool_window=w.pool_window,
+                        n_keep_head=w.keep_head, n_keep_tail=w.keep_tail)
+    assert torch.equal(idx[0], idx[1])
