@@ -785,3 +785,96 @@ def test_checkpoint_and_resume_is_bit_identical():
         R.retrieve_topk(bank, queries.to(DEV), w.T, w.k, i, scale=0.5, pool_window=w.pool_window,
                         n_keep_head=w.keep_head, n_keep_tail=w.keep_tail)
     assert torch.equal(idx[0], idx[1])
+
+
+def test_evict_seeded_random_shapes():
+    """Eighty seeded shapes of the cache compression (1 to 12 segments, 1 to 40,000 keys, budgets from
+    a handful to nearly everything, sink / recent rows from none to most of the budget, score
+    distributions from continuous to heavily tied, padded capacities so that vector and scalar key
+    loads both occur, with and without the position map and the kept-index output), each compared
+    bit for bit with the oracle's full sort.  Most take the one-launch form; shapes with many
+    segments take the block-per-segment or per-pass forms."""
+    import random
+    rnd = random.Random(20250602)
+    for case in range(80):
+        B = rnd.choice([1, 1, 2, 3]); Hkv = rnd.choice([1, 2, 4])
+        n = rnd.choice([1, 2, 7, 33, 500, 1023, 1024, 4095, 4096, 8191, 8192, 8193, 12000, 16385, 30000, 40000])
+        budget = max(1, min(n + rnd.choice([-1, 0, 5]), rnd.choice([1, 8, 100, n // 5 + 1, n // 2 + 1, n - 1, n])))
+        sink = rnd.choice([0, 0, 1, 4, budget // 3])
+        recent = rnd.choice([0, 0, 1, 4, budget // 3])
+        if sink + recent > budget or sink + recent > n:
+            sink, recent = 0, min(recent, budget, n) // 2
+        cap = n + rnd.choice([0, 1, 3, 4, 8])
+        d = rnd.choice([4, 8, 64])
+        dtype = rnd.choice([torch.float32, torch.bfloat16]) if d >= 8 else torch.float32
+        g = torch.Generator().manual_seed(case * 104729 + 7)
+        k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+        v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+        kind = rnd.choice(["uniform", "heavy_tail", "tied", "two_level", "constant", "signed"])
+        u = torch.rand(B, Hkv, cap, generator=g)
+        sc = {"uniform": u, "heavy_tail": torch.exp(8 * u) / 2981.0, "tied": (u * 7).floor() / 7,
+              "two_level": 1.0 + (u * 40).floor() * 2.0 ** -23, "constant": torch.full_like(u, 0.25),
+              "signed": (u - 0.5) * 3}[kind]
+        with_pos, with_kept = rnd.random() < 0.5, rnd.random() < 0.7
+        pos = torch.randint(0, 1 << 20, (B, Hkv, cap), generator=g, dtype=torch.int32) if with_pos else None
+        ref = oracle.evict_topk(k, v, sc, n, budget, sink, recent, cap_dst=budget, pos_src=pos)
+        kd = torch.zeros(B, Hkv, budget, d, dtype=dtype, device=DEV)
+        vd, sd = torch.zeros_like(kd), torch.zeros(B, Hkv, budget, device=DEV)
+        pd = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV) if with_pos else None
+        kept = torch.full((B, Hkv, budget), -1, dtype=torch.int32, device=DEV) if with_kept else None
+        status = "case %d: B %d Hkv %d n %d budget %d sink %d recent %d cap %d %s" % (
+            case, B, Hkv, n, budget, sink, recent, cap, kind)
+        n_kept = R.evict_topk(k.to(DEV), v.to(DEV), sc.to(DEV), kd, vd, sd, n, budget, sink, recent,
+                              pos_src=pos.to(DEV) if with_pos else None, pos_dst=pd, kept_idx=kept)
+        torch.cuda.synchronize()
+        assert n_kept == ref["n_kept"], status
+        if with_kept:
+            assert torch.equal(kept.cpu()[:, :, :n_kept], ref["kept_idx"][:, :, :n_kept]), status
+        assert torch.equal(kd.cpu()[:, :, :n_kept].view(torch.uint8), ref["k"][:, :, :n_kept].view(torch.uint8)), status
+        assert torch.equal(vd.cpu()[:, :, :n_kept].view(torch.uint8), ref["v"][:, :, :n_kept].view(torch.uint8)), status
+        assert torch.equal(sd.cpu()[:, :, :n_kept].double(), ref["score"][:, :, :n_kept]), status
+        if with_pos:
+            assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept]), status
+    assert R.device_error() == 0
+
+
+def test_retrieve_seeded_random_shapes():
+    """Forty seeded shapes of the retrieval (bank lengths on and off the tile grids, 1 to 64 queries,
+    row widths that take the tensor-core scan and ones that do not, fp32 and bf16, pooling windows 1
+    to 257 in both modes, forced head / tail rows, k from 1 to beyond N), each against the oracle
+    in full."""
+    import random
+    rnd = random.Random(20250603)
+    for case in range(40):
+        B = rnd.choice([1, 1, 2, 3])
+        N = rnd.choice([1, 5, 127, 128, 129, 1000, 4095, 4096, 4097, 9000, 20000])
+        E = rnd.choice([32, 64, 128, 192, 1024])
+        nq = rnd.choice([1, 2, 4, 8, 17, 64])
+        dtype = rnd.choice([torch.bfloat16, torch.bfloat16, torch.float32])
+        pool = rnd.choice([1, 3, 5, 21, 129, 257])
+        mode = rnd.choice(["max", "mean"])
+        k = rnd.choice([1, 8, 100, N // 3 + 1, N, N + 10])
+        keep_h = rnd.choice([0, 0, 1, 3]); keep_t = rnd.choice([0, 0, 2, 5])
+        if keep_h + keep_t > min(k, N):
+            keep_h = keep_t = 0
+        g = torch.Generator().manual_seed(case * 7907 + 3)
+        bank = torch.randn(B, N + rnd.choice([0, 3]), E, generator=g).to(dtype)
+        qs = torch.randn(B, nq, E, generator=g).to(dtype)
+        scale = 1.0 / E ** 0.5
+        status = "case %d: B %d N %d E %d nq %d %s pool %d %s k %d keep %d/%d" % (
+            case, B, N, E, nq, dtype, pool, mode, k, keep_h, keep_t)
+        p = dict(scale=scale, pool_window=pool, n_keep_head=keep_h, n_keep_tail=keep_t)
+        ref = oracle.retrieve_topk(bank, qs, N, k, pool_mode=mode, **p)
+        idx = torch.full((B, max(k, 1)), -1, dtype=torch.int32, device=DEV)
+        ts = torch.zeros(B, N, device=DEV)
+        pooled = torch.zeros(B, N, device=DEV)
+        n_out = R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx, token_score_out=ts, pooled_score_out=pooled,
+                                pool_mode=R.POOL_MEAN if mode == "mean" else R.POOL_MAX, **p)
+        torch.cuda.synchronize()
+        assert n_out == ref["n_out"], status
+        # bf16 products are exact in fp32 and the sums differ from fp64 only by fp32 rounding
+        assert_scores_close(ts, ref["ts"], 1.0)
+        assert_scores_close(pooled, ref["pooled"], 1.0)
+        for b in range(B):
+            assert_index_sets_match(idx[b, :n_out].cpu(), ref["idx"][b], ref["pooled"][b], rel=1e-4)
+    assert R.device_error() == 0
