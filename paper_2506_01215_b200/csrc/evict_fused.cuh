@@ -327,36 +327,14 @@ evict_fused_kernel(const EvictFusedArgs a) {
     for (int i = tid; i < a.lo; i += kSelThreads) out[i] = i;
     const int tail = a.n - a.hi;
     for (int i = tid; i < tail; i += kSelThreads) out[a.lo + i] = a.hi + i;
-    publish_phase(a.flags + (size_t)blockIdx.x * a.nb, a.epoch, 3);   // the segment's first flag stands for it
+    publish_phase(a.flags + blockIdx.x, a.epoch, 3);   // no selection blocks in this mode: flag s stands for segment s
   }
 
   // compaction: wait for every kept list, then stream the rows
   if (a.m > 0) {
     if (!wait_flags(a.flags, n_sel_blocks, nullptr, a.epoch, 3, abort_word, a.wait_cycles, 100, a.dev_status)) return;
   } else {
-    for (int s0 = 0; s0 < a.segs; s0 += kSelThreads) {   // flag 0 of every segment
-      const int s = s0 + tid;
-      __shared__ int bad;
-      if (tid == 0) bad = 0;
-      __syncthreads();
-      if (s < a.segs) {
-        const long long t0 = clock64();
-        for (;;) {
-          const unsigned long long v = ld_acquire_u64(a.flags + (size_t)s * a.nb);
-          if ((v & ~7ull) == a.epoch && (unsigned)(v & 7ull) >= 3u) break;
-          __nanosleep(100);
-          if (ld_acquire_u64(abort_word) == a.epoch || clock64() - t0 > a.wait_cycles) {
-            st_release_u64(abort_word, a.epoch);
-            report_device_error(a.dev_status, REFORM_DEV_TIMEOUT);
-            bad = 1;
-            break;
-          }
-        }
-      }
-      __syncthreads();
-      if (bad) return;
-      __syncthreads();
-    }
+    if (!wait_flags(a.flags, a.segs, nullptr, a.epoch, 3, abort_word, a.wait_cycles, 100, a.dev_status)) return;
   }
   constexpr int LANES = 4;
   constexpr int ROWS = kSelThreads / LANES;
