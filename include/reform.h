@@ -165,8 +165,18 @@ int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream);
  *   pos_dst      optional; kept_idx [B,Hkv,budget] int32 out, optional
  * Rows [0, n_kept) of the destinations are written, n_kept = min(n_keys,
  * budget), also stored to *n_kept_host (host int32, optional) before return.
- * Destinations must not overlap sources.  n_sink + n_recent > budget, or
- * n_kept > cap_dst, is REFORM_ERR_INVALID_ARG.
+ * n_sink + n_recent > budget, or n_kept > cap_dst, is REFORM_ERR_INVALID_ARG.
+ *
+ * In place: the destinations may BE the sources -- k_dst == k_src, v_dst ==
+ * v_src, score_dst == score_src, pos_dst == pos_src, cap_dst == cap_src, all
+ * of them or none (a mixture, or any other overlap, is outside the contract;
+ * equal pointers in a mixture are REFORM_ERR_INVALID_ARG).  The kept rows then
+ * move down inside their own buffers and a layer needs one K/V buffer instead
+ * of two.  In place needs rows of at most 256 bytes and a shape whose
+ * selection blocks fit the device at once (segments up to 262,144 keys, about
+ * a device's worth of 8,192-key blocks per call); otherwise the call returns
+ * REFORM_ERR_UNSUPPORTED and nothing is launched.  The workspace needs no
+ * clearing between calls.
  * ------------------------------------------------------------------------ */
 typedef struct reform_evict_params {
   size_t struct_size;

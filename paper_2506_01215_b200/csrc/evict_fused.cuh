@@ -21,6 +21,13 @@
 //   -- hand-off 3: the kept lists of all segments are complete --
 // Then every block of the grid streams kept rows (128-bit loads and stores).
 //
+// In place (destinations == sources): kept rows only ever move down (kept[r] >= r, ascending), so
+// the ranks are taken in waves of as many rows as the grid can hold in registers at once: every
+// block loads its rows of the wave, all blocks meet (one more flag per block), then every block
+// stores.  A wave's stores land in rank positions [w R, (w+1) R) of each segment; every row that
+// still has to be read from there belongs to this wave or an earlier one and is in registers by
+// then, and later waves read from beyond (w+1) R.
+//
 // Hand-offs are 64-bit flags, one per selection block, that carry the call's
 // epoch and the phase reached; a stale flag from an earlier call (or whatever
 // the workspace held before) never matches the epoch, so the workspace needs no
@@ -39,6 +46,9 @@ constexpr int kEvPerThread = 8;            // consecutive keys a thread holds in
 constexpr int kEvTile = kSelThreads * kEvPerThread;   // keys per selection block
 constexpr int kEvMaxBlocksPerSeg = 32;     // slices each block has to add up (segments up to 262,144 keys)
 constexpr long long kEvWaitCycles = 400000000LL;  // about 0.2 s; real waits are microseconds
+constexpr unsigned long long kEvPhaseMask = 0xFFull;   // a flag is (epoch with these bits clear) | phase
+constexpr int kEvMaxGrid = 1024;           // blocks a launch may have (one flag each for the in-place copy)
+constexpr int kEvMaxWaves = 200;           // in-place copy: phases 4 .. 4 + waves - 1 must fit the phase field
 
 struct EvictFusedArgs {
   // selection
@@ -50,9 +60,10 @@ struct EvictFusedArgs {
   int segs, nb;
   uint32_t* slices;            // [segs][nb][kSelBins]
   uint32_t* cand;              // [segs][n]
-  unsigned long long* flags;   // [segs * nb] one flag per selection block, then the abort word, then a slot nothing writes
+  unsigned long long* flags;   // [segs * nb] one flag per selection block, the abort word, a slot nothing writes, [kEvMaxGrid] one flag per block of the grid
   int expect_extra;            // diagnostic: the first hand-off also waits for the slot nothing writes (0 in normal use)
-  unsigned long long epoch;    // already shifted: phase goes into the low 3 bits
+  unsigned long long epoch;    // low 8 bits clear: the phase goes there
+  int in_place;                // destinations are the sources: rows move down inside their own buffers
   long long wait_cycles;
   // compaction
   const uint4* k_src;
@@ -78,7 +89,7 @@ inline EvictFusedLayout evict_fused_layout(int segs, int n) {
   if (L.nb < 1) L.nb = 1;
   size_t off = 0;
   L.flags = off;
-  off += align_up(sizeof(unsigned long long) * ((size_t)segs * L.nb + 2), 256);
+  off += align_up(sizeof(unsigned long long) * ((size_t)segs * L.nb + 2 + kEvMaxGrid), 256);
   L.slices = off;
   off += align_up(sizeof(uint32_t) * (size_t)segs * L.nb * kSelBins, 256);
   L.cand = off;
@@ -112,7 +123,7 @@ __device__ __forceinline__ bool wait_flags(const unsigned long long* flags, int 
     const unsigned long long* f = i < count ? flags + i : extra;
     for (uint32_t it = 0;; ++it) {
       const unsigned long long v = ld_acquire_u64(f);
-      if ((v & ~7ull) == epoch && (unsigned)(v & 7ull) >= phase) break;
+      if ((v & ~kEvPhaseMask) == epoch && (unsigned)(v & kEvPhaseMask) >= phase) break;
       if (sleep_ns) __nanosleep(sleep_ns);
       if ((it & 15u) == 15u || sleep_ns) {
         if (ld_acquire_u64(abort_word) == epoch || *(volatile int*)&wf_failed) { wf_failed = 1; break; }
@@ -339,6 +350,53 @@ evict_fused_kernel(const EvictFusedArgs a) {
   constexpr int LANES = 4;
   constexpr int ROWS = kSelThreads / LANES;
   const int lane = tid % LANES, sub = tid / LANES;
+  if (a.in_place) {   // rows of at most 16 chunks (checked by the launcher): four per lane and tensor
+    unsigned long long* gflags = abort_word + 2;
+    const int per_wave = (int)gridDim.x * ROWS;
+    const int Rw = per_wave / a.segs > 0 ? per_wave / a.segs : 1;   // ranks per segment and wave
+    const int waves = (a.n_kept + Rw - 1) / Rw;
+    const int item = (int)blockIdx.x * ROWS + sub;
+    const int s = item / Rw;
+    for (int w = 0; w < waves; ++w) {
+      const int rank = w * Rw + item % Rw;
+      const bool live = s < a.segs && rank < a.n_kept;
+      uint4 kk[4], vv[4];
+      float sc = 0.f;
+      int32_t ps = 0;
+      long long dn = 0;
+      if (live) {
+        const int j = __ldcg(a.out + (long long)s * a.out_stride + rank);
+        const long long so = ((long long)s * a.cap_src + j) * a.vec;
+        dn = ((long long)s * a.cap_dst + rank) * a.vec;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (lane + u * LANES < a.vec) {
+            kk[u] = __ldcg(a.k_src + so + lane + u * LANES);
+            vv[u] = __ldcg(a.v_src + so + lane + u * LANES);
+          }
+        if (lane == 0) {
+          sc = __ldcg(a.score_src + (long long)s * a.cap_src + j);
+          if (a.pos_dst) ps = __ldcg(a.pos_src + (long long)s * a.cap_src + j);
+        }
+      }
+      __threadfence();   // every thread's loads of this wave have been performed before the block says so
+      publish_phase(gflags + blockIdx.x, a.epoch, 4 + w);
+      if (!wait_flags(gflags, (int)gridDim.x, nullptr, a.epoch, 4 + w, abort_word, a.wait_cycles, 0, a.dev_status)) return;
+      if (live) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (lane + u * LANES < a.vec) {
+            __stcg(a.k_dst + dn + lane + u * LANES, kk[u]);
+            __stcg(a.v_dst + dn + lane + u * LANES, vv[u]);
+          }
+        if (lane == 0) {
+          a.score_dst[(long long)s * a.cap_dst + rank] = sc;
+          if (a.pos_dst) a.pos_dst[(long long)s * a.cap_dst + rank] = ps;
+        }
+      }
+    }
+    return;
+  }
   const long long total = (long long)a.segs * a.n_kept;
   for (long long r = (long long)blockIdx.x * ROWS + sub; r < total; r += (long long)gridDim.x * ROWS) {
     const int s = (int)(r / a.n_kept), rank = (int)(r % a.n_kept);
@@ -389,17 +447,32 @@ inline bool evict_fused_applies(int segs, int n, size_t workspace_bytes, size_t 
   const EvictFusedLayout L = evict_fused_layout(segs, n);
   if (L.nb > kEvMaxBlocksPerSeg) return false;
   if (workspace_bytes < L.total + kept_bytes) return false;
-  return (long long)segs * L.nb <= evict_fused_capacity();
+  const int capacity = evict_fused_capacity() < kEvMaxGrid ? evict_fused_capacity() : kEvMaxGrid;
+  return (long long)segs * L.nb <= capacity;
 }
 
-inline int launch_evict_fused(EvictFusedArgs a, cudaStream_t st) {
-  const int capacity = evict_fused_capacity();
+// In-place compaction holds a wave of rows in registers: rows of at most 256 bytes, and few enough
+// waves for the phase field.
+inline bool evict_fused_in_place_ok(int segs, int n_kept, int vec, int grid) {
+  if (vec > 16) return false;
+  const int per_wave = grid * (kSelThreads / 4);
+  const int Rw = per_wave / segs > 0 ? per_wave / segs : 1;
+  return (n_kept + Rw - 1) / Rw <= kEvMaxWaves;
+}
+
+inline int evict_fused_grid(const EvictFusedArgs& a) {
+  const int capacity = evict_fused_capacity() < kEvMaxGrid ? evict_fused_capacity() : kEvMaxGrid;
   const long long rows = (long long)a.segs * a.n_kept;
   long long want = (rows + (kSelThreads / 4) - 1) / (kSelThreads / 4);   // blocks that find a row to move
   const long long sel_blocks = (long long)a.segs * a.nb;
   if (want < sel_blocks) want = sel_blocks;
   if (want < a.segs) want = a.segs;
-  const int grid = (int)(want < capacity ? want : capacity);
+  return (int)(want < capacity ? want : capacity);
+}
+
+inline int launch_evict_fused(EvictFusedArgs a, cudaStream_t st) {
+  const int grid = evict_fused_grid(a);
+  if (a.in_place && !evict_fused_in_place_ok(a.segs, a.n_kept, a.vec, grid)) return REFORM_ERR_UNSUPPORTED;
   void* args[] = {&a};
   cudaError_t e = cudaLaunchCooperativeKernel((const void*)evict_fused_kernel, dim3(grid), dim3(kSelThreads), args, 0, st);
   if (e != cudaSuccess) {

@@ -244,6 +244,11 @@ int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream) {
 
 /* ---------------------------------------------------------------- evict */
 
+static bool evict_in_place(const reform_evict_params* p) {
+  return p->k_src == p->k_dst && p->v_src == p->v_dst && p->score_src == p->score_dst &&
+         p->pos_src == p->pos_dst && p->cap_src == p->cap_dst;
+}
+
 static int validate_evict(const reform_evict_params* p) {
   if (!p || p->struct_size != sizeof(reform_evict_params)) return REFORM_ERR_INVALID_ARG;
   if (!dtype_ok(p->dtype)) return REFORM_ERR_UNSUPPORTED;
@@ -261,8 +266,10 @@ static int validate_evict(const reform_evict_params* p) {
   if (!aligned16(p->k_src) || !aligned16(p->v_src) || !aligned16(p->k_dst) || !aligned16(p->v_dst) ||
       !aligned16(p->score_src) || !aligned16(p->score_dst) || !aligned16(p->kept_idx))
     return REFORM_ERR_INVALID_ARG;
-  if (p->k_src == p->k_dst || p->v_src == p->v_dst || p->score_src == p->score_dst)
-    return REFORM_ERR_INVALID_ARG;
+  // in place means all of K, V, score (and position) in place, with one capacity; otherwise none
+  const bool any_same = p->k_src == p->k_dst || p->v_src == p->v_dst || p->score_src == p->score_dst ||
+                        (p->pos_src && p->pos_src == p->pos_dst);
+  if (any_same && !evict_in_place(p)) return REFORM_ERR_INVALID_ARG;
   return REFORM_OK;
 }
 
@@ -305,8 +312,11 @@ static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need,
   }
   const int row_bytes = (int)(p->d * elem_size(p->dtype));
   const size_t kept_bytes = p->kept_idx ? 0 : evict_kept_bytes(p);
+  const bool in_place = evict_in_place(p);
   const bool many_short = p->n_keys <= kSelBlockMaxN && segs >= kSelBlockMinSegs;  // one block per segment wins
-  if (!many_short && evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes)) {
+  if (in_place && !evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes))
+    return REFORM_ERR_UNSUPPORTED;   // only the one-launch form can move rows inside their own buffers
+  if ((in_place || !many_short) && evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes)) {
     // one cooperative launch: selection with two hand-offs, then the compaction
     const EvictFusedLayout F = evict_fused_layout(segs, p->n_keys);
     EvictFusedArgs a;
@@ -324,7 +334,8 @@ static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need,
     a.cand = reinterpret_cast<uint32_t*>(ws + F.cand);
     a.flags = reinterpret_cast<unsigned long long*>(ws + F.flags);
     a.expect_extra = expect_extra;
-    a.epoch = next_epoch();
+    a.epoch = next_epoch() << 5;
+    a.in_place = in_place ? 1 : 0;
     a.wait_cycles = wait_cycles;
     a.k_src = (const uint4*)p->k_src;
     a.v_src = (const uint4*)p->v_src;

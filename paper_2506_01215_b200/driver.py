@@ -16,8 +16,9 @@ class LayerCache:
 
     ``n_buffers`` buffer sets of shape [B,Hkv,cap,d] are used round-robin: the
     chunk step of recurrence step s reads set s % n_buffers and the eviction
-    writes the compacted rows into set (s+1) % n_buffers (source and
-    destination of reform_evict_topk must differ).
+    writes the compacted rows into set (s+1) % n_buffers.  With ``n_buffers = 1``
+    the eviction runs in place (destinations are the sources) and the layer
+    holds one K/V buffer instead of two.
     """
 
     def __init__(self, B, Hkv, d, cap, budget, n_sink, n_recent, dtype, device, n_buffers=2):

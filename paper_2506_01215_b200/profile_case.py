@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--simt", action="store_true")
     ap.add_argument("--no-score", action="store_true", help="chunk_step without the key-score pass")
     ap.add_argument("--rope", action="store_true", help="chunk_step on un-rotated operands (REFORM_ROPE)")
+    ap.add_argument("--in-place", action="store_true", help="evict: destinations are the sources")
     ap.add_argument("--graph", action="store_true",
                     help="capture the call in a CUDA graph and time its replays (device time without the "
                          "host's launch cost)")
@@ -55,7 +56,7 @@ def main():
             (R.ROPE if a.rope else 0)
         fn = lambda: R.chunk_step(q, k, v, out, score, w.budget, w.window, lse=lse, flags=flags)
     elif a.op == "evict":
-        kd, vd, sd = torch.empty_like(k), torch.empty_like(v), torch.empty_like(score)
+        kd, vd, sd = (k, v, score) if a.in_place else (torch.empty_like(k), torch.empty_like(v), torch.empty_like(score))
         kept = torch.empty(wb.B, wb.Hkv, wb.budget, dtype=torch.int32, device=dev)
         fn = lambda: R.evict_topk(k, v, score, kd, vd, sd, wb.cap, wb.budget, wb.n_sink, wb.n_recent,
                                   kept_idx=kept)

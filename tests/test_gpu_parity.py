@@ -878,3 +878,62 @@ def test_retrieve_seeded_random_shapes():
         for b in range(B):
             assert_index_sets_match(idx[b, :n_out].cpu(), ref["idx"][b], ref["pooled"][b], rel=1e-4)
     assert R.device_error() == 0
+
+
+@pytest.mark.parametrize("B,Hkv,d,n_keys,budget,sink,recent,dtype", [
+    (1, 2, 64, 1536, 512, 32, 32, torch.float32),      # Tiny's shapes
+    (1, 8, 128, 40960, 8192, 256, 256, torch.bfloat16),  # config 2: 65,536 rows, more than one wave of the copy
+    (4, 8, 128, 20480, 4096, 256, 256, torch.bfloat16),  # config 5: 32 segments
+    (2, 3, 8, 9001, 9000, 0, 0, torch.float32),        # nearly everything kept: rows barely move
+    (1, 1, 32, 300, 40, 16, 24, torch.bfloat16),       # forced rows only
+    (1, 2, 64, 100, 128, 8, 8, torch.float32),         # under budget: every row stays where it is
+])
+def test_evict_in_place_matches_oracle(B, Hkv, d, n_keys, budget, sink, recent, dtype):
+    """Destinations == sources: the kept rows move down inside their own buffers (one K/V buffer per
+    layer instead of two).  Same bits as the oracle's out-of-place result in rows [0, n_kept)."""
+    g = torch.Generator().manual_seed(n_keys + budget)
+    cap = n_keys + 5
+    k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    sc = torch.rand(B, Hkv, cap, generator=g)
+    sc[:, :, ::5] = (sc[:, :, ::5] * 8).floor() / 8
+    pos = torch.randint(0, 1 << 20, (B, Hkv, cap), generator=g, dtype=torch.int32)
+    ref = oracle.evict_topk(k, v, sc, n_keys, budget, sink, recent, cap_dst=cap, pos_src=pos)
+    kd, vd, sd, pd = k.to(DEV), v.to(DEV), sc.to(DEV), pos.to(DEV)
+    kept = torch.full((B, Hkv, budget), -1, dtype=torch.int32, device=DEV)
+    n_kept = R.evict_topk(kd, vd, sd, kd, vd, sd, n_keys, budget, sink, recent, pos_src=pd, pos_dst=pd,
+                          kept_idx=kept)
+    torch.cuda.synchronize()
+    assert R.device_error() == 0
+    assert n_kept == ref["n_kept"]
+    assert torch.equal(kept.cpu()[:, :, :n_kept], ref["kept_idx"][:, :, :n_kept])
+    assert torch.equal(kd.cpu()[:, :, :n_kept].view(torch.uint8), ref["k"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(vd.cpu()[:, :, :n_kept].view(torch.uint8), ref["v"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(sd.cpu()[:, :, :n_kept].double(), ref["score"][:, :, :n_kept])
+    assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept])
+    # rows past the keys in use are untouched
+    assert torch.equal(kd.cpu()[:, :, n_keys:], k[:, :, n_keys:])
+
+
+def test_evict_in_place_recurrence_equals_ping_pong():
+    """Tiny's 8 chunk steps through the driver with one buffer set per layer (in-place compaction)
+    against the same recurrence with two (out of place): the same outputs and the same cache, bit
+    for bit, after every step."""
+    w = synth.WORKLOADS["tiny"]
+    two = LayerCache(w.B, w.Hkv, w.d, w.cap, w.budget, w.n_sink, w.n_recent, w.dtype, DEV)
+    one = LayerCache(w.B, w.Hkv, w.d, w.cap, w.budget, w.n_sink, w.n_recent, w.dtype, DEV, n_buffers=1)
+    out2 = torch.zeros(w.B, w.Hq, w.Lc, w.d, device=DEV)
+    out1 = torch.zeros_like(out2)
+    for step in range(w.steps):
+        q, kc, vc = (t.to(DEV) for t in synth.chunk_qkv(w, 0, step))
+        for cache, out in ((two, out2), (one, out1)):
+            cache.write_chunk(kc, vc)
+            cache.attend(q, out, w.window)
+            cache.evict()
+        n = one.n_cache
+        assert n == two.n_cache and one.cur == 0
+        assert torch.equal(out1, out2)
+        assert torch.equal(one.k[0][:, :, :n], two.k[two.cur][:, :, :n])
+        assert torch.equal(one.v[0][:, :, :n], two.v[two.cur][:, :, :n])
+        assert torch.equal(one.score[0][:, :, :n], two.score[two.cur][:, :, :n])
+        assert torch.equal(one.kept_idx, two.kept_idx)

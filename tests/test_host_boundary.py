@@ -128,9 +128,19 @@ def test_chunk_step_size_query_validates_shapes():
 @pytest.mark.parametrize("kw", [
     dict(n_sink=20, n_recent=20), dict(n_keys=200), dict(cap_dst=16), dict(k_dst=FAKE),
     dict(pos_src=FAKE), dict(score_src=None), dict(budget=-1),
+    # in place means everything in place and one capacity: a mixture is refused
+    dict(k_dst=FAKE, v_dst=FAKE, score_dst=FAKE),
+    dict(k_dst=FAKE, v_dst=FAKE, score_dst=FAKE, cap_dst=128, pos_src=FAKE, pos_dst=FAKE + 64),
 ])
 def test_evict_rejects_bad_arguments(kw):
     assert R.lib().reform_evict_topk(ctypes.byref(_evict(**kw)), None) == R.ERR_INVALID_ARG
+
+
+def test_evict_in_place_is_accepted_by_the_validation():
+    """All destinations equal to their sources with one capacity passes validation (it then asks for
+    its workspace like any other call)."""
+    p = _evict(k_dst=FAKE, v_dst=FAKE, score_dst=FAKE, cap_dst=128)
+    assert R.lib().reform_evict_topk(ctypes.byref(p), None) == R.ERR_WORKSPACE
 
 
 def test_evict_reports_n_kept_and_needs_workspace():
