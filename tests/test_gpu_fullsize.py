@@ -63,6 +63,40 @@ def test_chunk_step_llama8b_full_size_spot_check():
     _chunk_step_spot_check("llama8b_128k", 0, groups=[0, 5])
 
 
+def test_chunk_step_with_rope_full_size_spot_check():
+    """Config 2's step with the rotary embedding applied inside the call (un-rotated q and k in,
+    positions 0 .. 40,959 for the keys and 8,192 .. 40,959 for the queries): sampled rows of one KV
+    group against the oracle rotating in fp64, and the whole group's score row."""
+    w = synth.WORKLOADS["llama8b_128k"]
+    G = w.Hq // w.Hkv
+    g = 6
+    q, kc, vc = synth.chunk_qkv(w, 0, 2, device=DEV)
+    k0, v0, s0 = synth.cache_state(w, 1, device=DEV)
+    k = torch.cat([k0, kc], 2).contiguous()
+    v = torch.cat([v0, vc], 2).contiguous()
+    carry = torch.cat([s0, torch.zeros(w.B, w.Hkv, w.Lc, device=DEV)], 2).contiguous()
+    score = carry.clone()
+    out = torch.empty_like(q)
+    lse = torch.empty(q.shape[:3], dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    R.chunk_step(q, k, v, out, score, w.budget, w.window, lse=lse, flags=R.SCORE_ACCUMULATE | R.ROPE,
+                 rope_theta=500000.0, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and R.device_error() == 0
+    n = w.cap
+    new = score[:, :, :n].double().sum(-1) - carry[:, :, :w.budget].double().sum(-1)
+    assert torch.allclose(new, torch.full_like(new, float(w.window * G)), rtol=1e-3)
+    rows = _sample_rows(w.Lc, 11)
+    qs = oracle.rope(q[:, g * G:(g + 1) * G].cpu().contiguous(), 0, w.Lc, w.budget, base=500000.0)
+    ks = oracle.rope(k[:, g:g + 1].cpu().contiguous(), 0, n, 0, base=500000.0)
+    vs = v[:, g:g + 1].cpu().contiguous()
+    o_ref, l_ref = oracle.attention(qs, ks, vs, w.budget, rows=rows)
+    assert_outputs_close(out[:, g * G:(g + 1) * G][:, :, rows], o_ref, w.dtype)
+    assert (lse[:, g * G:(g + 1) * G][:, :, rows].cpu().double() - l_ref).abs().max() < 3e-3
+    s_ref = oracle.key_scores(qs, ks, w.budget, w.window, score_in=carry[:, g:g + 1].cpu(), accumulate=True)
+    assert_scores_close(score[:, g:g + 1, :n], s_ref[:, :, :n], w.window * G / n)
+
+
 def test_chunk_step_mistral_batched_full_size_spot_check():
     """Config 5: batch of 4, chunk 16,384 over a 4,096-row cache."""
     _chunk_step_spot_check("mistral7b_4x256k", 2, groups=[3])
