@@ -230,3 +230,23 @@ def test_empty_inputs_are_accepted_and_launch_nothing():
     assert L.reform_gather(ctypes.byref(_gather(B=0)), None) == R.OK
     assert L.reform_rope(ctypes.byref(_rope(rows=0)), None) == R.OK
     assert R.kernel_launch_count() == n0
+
+
+def test_header_is_plain_c_and_struct_sizes_match_the_binding(tmp_path):
+    """include/reform.h compiles as C99 on its own, and every params struct has the size the ctypes
+    binding gives it (field order, widths and padding agree)."""
+    import os
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    names = [("reform_chunk_params", R.ChunkParams), ("reform_evict_params", R.EvictParams),
+             ("reform_embed_params", R.EmbedParams), ("reform_retrieve_params", R.RetrieveParams),
+             ("reform_gather_params", R.GatherParams), ("reform_rope_params", R.RopeParams),
+             ("reform_head_sel", R.HeadSel)]
+    src = tmp_path / "sizes.c"
+    src.write_text('#include <stdio.h>\n#include "reform.h"\nint main(void) {\n' +
+                   "".join(f'  printf("%zu\\n", sizeof({n}));\n' for n, _ in names) + "  return 0;\n}\n")
+    exe = tmp_path / "sizes"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror",
+                           "-I", os.path.join(root, "include"), str(src), "-o", str(exe)])
+    sizes = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    assert sizes == [ctypes.sizeof(t) for _, t in names]
