@@ -20,7 +20,8 @@
  *   - All tensor pointers are DEVICE pointers unless a field says "host".
  *     The caller owns every buffer; the library allocates nothing and keeps
  *     no pointer after the call returns.  Its global state is: a per-thread
- *     record of the last CUDA error, a launch counter, one error word per
+ *     record of the last CUDA error and of the last selection's launch form
+ *     (reform_debug_last_path), a launch counter, one error word per
  *     device (reform_device_error) and, per device, the fixed scratch array
  *     of reform_evict_topk_static (REFORM_EVICT_STATIC_BYTES).
  *   - Work is enqueued on the caller's stream and the call returns without
@@ -427,6 +428,16 @@ int reform_version(void);
 /* Number of kernels this library has launched from the calling process since
  * load (monotonic; for accounting in benchmarks). */
 long long reform_kernel_launch_count(void);
+/* Which launch form the last reform_evict_topk (or _static) or reform_retrieve_topk call made by
+ * this thread chose for its selection (diagnostic; the results do not depend on it). */
+enum {
+  REFORM_PATH_NONE = 0,        /* no such call yet, or nothing to select */
+  REFORM_PATH_CLUSTER = 1,     /* one thread-block cluster per segment, one launch */
+  REFORM_PATH_COOPERATIVE = 2, /* one cooperative launch over global-memory hand-offs */
+  REFORM_PATH_PER_SEGMENT = 3, /* one block per segment (many short segments), then the row copy */
+  REFORM_PATH_PER_PASS = 4     /* one launch per radix pass, then the row copy */
+};
+int reform_debug_last_path(void);
 
 #ifdef __cplusplus
 }

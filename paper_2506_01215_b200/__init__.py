@@ -87,6 +87,7 @@ EXPORTS = (
     "reform_embed_append", "reform_retrieve_topk",
     "reform_retrieve_topk_workspace_size", "reform_gather", "reform_rope", "reform_status_string",
     "reform_last_cuda_error", "reform_device_error", "reform_version", "reform_kernel_launch_count",
+    "reform_debug_last_path",
 )
 
 _lib = None
@@ -133,6 +134,7 @@ def lib() -> ctypes.CDLL:
         L.reform_device_error.restype = ctypes.c_int
         L.reform_version.restype = ctypes.c_int
         L.reform_kernel_launch_count.restype = ctypes.c_longlong
+        L.reform_debug_last_path.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -149,6 +151,15 @@ def device_error(clear: bool = True) -> int:
 
 def kernel_launch_count() -> int:
     return int(lib().reform_kernel_launch_count())
+
+
+PATH_NONE, PATH_CLUSTER, PATH_COOPERATIVE, PATH_PER_SEGMENT, PATH_PER_PASS = 0, 1, 2, 3, 4
+
+
+def debug_last_path() -> int:
+    """reform_debug_last_path: the launch form (PATH_*) the calling thread's last evict_topk or
+    retrieve_topk chose for its selection."""
+    return int(lib().reform_debug_last_path())
 
 
 def _dtype_code(t: torch.Tensor) -> int:

@@ -26,6 +26,7 @@ inline int num_sms() {
 
 // Per-thread record of the last failing CUDA call and a process-wide launch counter.
 extern thread_local int g_last_cuda_error;
+extern thread_local int g_last_path;   // REFORM_PATH_* of this thread's last selection
 void count_launch(int n = 1);
 
 inline int check_launch() {

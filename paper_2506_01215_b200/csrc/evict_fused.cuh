@@ -152,27 +152,6 @@ __device__ __forceinline__ void publish_phase(unsigned long long* flag, unsigned
   }
 }
 
-// Bin walk over a shared-memory histogram of kSelBins bins from the top: the bin in which the
-// running count reaches `remaining`, and how many are still to take inside it.  All threads get
-// the same answer.  result: 2 uints of shared memory; scratch: 33.
-__device__ __forceinline__ void find_bin_shared(const uint32_t* hist, uint32_t remaining, uint32_t* scratch,
-                                                uint32_t* result, uint32_t& bin_out, uint32_t& rem_out) {
-  const int b0 = kSelBins - 1 - 2 * (int)threadIdx.x;
-  const uint32_t c0 = hist[b0], c1 = hist[b0 - 1];
-  uint32_t total;
-  const uint32_t before = block_excl_scan(c0 + c1, scratch, total);
-  if (threadIdx.x == 0) { result[0] = kSelBins - 1; result[1] = 0; }
-  __syncthreads();
-  if (before < remaining && remaining <= before + c0 + c1) {
-    if (remaining <= before + c0) { result[0] = b0; result[1] = remaining - before; }
-    else { result[0] = b0 - 1; result[1] = remaining - before - c0; }
-  }
-  __syncthreads();
-  bin_out = result[0];
-  rem_out = result[1];
-  __syncthreads();
-}
-
 constexpr int kEvCandSmem = 8192;   // candidates of a segment staged in shared memory when they fit
 
 // key i of a segment's candidate list: from shared memory if the list was staged there

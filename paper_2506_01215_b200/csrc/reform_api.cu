@@ -11,6 +11,7 @@
 #include "rope.cuh"
 #include "select.cuh"
 #include "evict_fused.cuh"
+#include "select_cluster.cuh"
 #include "retrieve.cuh"
 #include "chunk_simt.cuh"
 #if !defined(REFORM_NO_SM100) && !__has_include("chunk_sm100.cuh")
@@ -24,6 +25,7 @@
 
 namespace reform {
 thread_local int g_last_cuda_error = 0;
+thread_local int g_last_path = REFORM_PATH_NONE;   // launch form of this thread's last selection (diagnostic)
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -291,12 +293,14 @@ size_t reform_evict_topk_workspace_size(const reform_evict_params* p) {
 }
 
 // need: the workspace size the entry point insists on.  wait_cycles / expect_extra: limits of the
-// hand-off waits of the one-launch form (diagnostic entry point; kEvWaitCycles and 0 otherwise).
+// hand-off waits of the cooperative one-launch form (diagnostic entry point, which also rules out the
+// cluster form, whose barriers are the hardware's; kEvWaitCycles and 0 otherwise).
 static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need, long long wait_cycles,
                      int expect_extra) {
   const int n_kept = p->n_keys < p->budget ? p->n_keys : p->budget;
   if (p->n_kept_host) *p->n_kept_host = n_kept;
   const int segs = p->B * p->Hkv;
+  g_last_path = REFORM_PATH_NONE;
   if (segs == 0 || n_kept == 0) return REFORM_OK;
   if (!p->workspace || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
     return REFORM_ERR_WORKSPACE;
@@ -314,8 +318,42 @@ static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need,
   const size_t kept_bytes = p->kept_idx ? 0 : evict_kept_bytes(p);
   const bool in_place = evict_in_place(p);
   const bool many_short = p->n_keys <= kSelBlockMaxN && segs >= kSelBlockMinSegs;  // one block per segment wins
+  if (expect_extra == 0 && (in_place ? row_bytes <= 256 : !many_short)) {
+    // one cluster per segment: selection and compaction in one launch, no workspace but the kept list.
+    // Taken in place always, and otherwise when the clusters run in one wave on enough blocks to
+    // stream the kept rows at the device's rate (the cooperative form below spreads the copy over
+    // the whole device whatever the number of segments).
+    const ClusterCapacity& cap = cluster_select_capacity<1>(cluster_sel_smem_bytes(false, 0, 0));
+    const int c = cluster_select_size(segs, p->n_keys, cap);
+    if (c && (in_place || (cluster_select_one_wave(segs, c, cap) && segs * c >= kClMinBlocksForCopy))) {
+      ClusterSelArgs a = {};
+      a.vals = p->score_src;
+      a.stride = p->cap_src;
+      a.n = p->n_keys;
+      a.lo = lo;
+      a.hi = hi;
+      a.m = m;
+      a.out = p->kept_idx ? p->kept_idx : reinterpret_cast<int32_t*>(ws);
+      a.out_stride = p->budget;
+      a.k_src = (const uint4*)p->k_src;
+      a.v_src = (const uint4*)p->v_src;
+      a.k_dst = (uint4*)p->k_dst;
+      a.v_dst = (uint4*)p->v_dst;
+      a.score_src = p->score_src;
+      a.score_dst = p->score_dst;
+      a.pos_src = p->pos_src;
+      a.pos_dst = p->pos_dst;
+      a.n_kept = n_kept;
+      a.cap_src = p->cap_src;
+      a.cap_dst = p->cap_dst;
+      a.vec = row_bytes / 16;
+      a.in_place = in_place ? 1 : 0;
+      g_last_path = REFORM_PATH_CLUSTER;
+      return launch_cluster_select<1>(a, segs, c, st);
+    }
+  }
   if (in_place && !evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes))
-    return REFORM_ERR_UNSUPPORTED;   // only the one-launch form can move rows inside their own buffers
+    return REFORM_ERR_UNSUPPORTED;   // only the one-launch forms can move rows inside their own buffers
   if ((in_place || !many_short) && evict_fused_applies(segs, p->n_keys, p->workspace_bytes, kept_bytes)) {
     // one cooperative launch: selection with two hand-offs, then the compaction
     const EvictFusedLayout F = evict_fused_layout(segs, p->n_keys);
@@ -350,6 +388,7 @@ static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need,
     a.cap_dst = p->cap_dst;
     a.vec = row_bytes / 16;
     a.dev_status = p->dev_status;
+    g_last_path = REFORM_PATH_COOPERATIVE;
     return launch_evict_fused(a, st);
   }
   SelLayout L = sel_layout(segs, p->n_keys);
@@ -519,6 +558,7 @@ size_t reform_retrieve_topk_workspace_size(const reform_retrieve_params* p) {
 int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream) {
   int rc = validate_retrieve(p);
   if (rc != REFORM_OK) return rc;
+  g_last_path = REFORM_PATH_NONE;
   if (p->B == 0 || p->N == 0 || p->k == 0) return REFORM_OK;
   size_t need = reform_retrieve_topk_workspace_size(p);
   if (!p->workspace || p->workspace_bytes < need || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
@@ -551,6 +591,28 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
     a.lo = p->n_keep_head;
     a.hi = (int)p->N - p->n_keep_tail;
     a.m = p->k - p->n_keep_head - p->n_keep_tail;
+  }
+  {
+    // banks of up to 16 x 8192 tokens: pooling and selection by one cluster per sequence
+    const int radius = (p->pool_window - 1) / 2;
+    const ClusterCapacity& cap = cluster_select_capacity<0>(cluster_sel_smem_bytes(true, kClTile, radius));
+    const int c = cluster_select_size(p->B, p->N, cap);
+    if (c && cluster_select_one_wave(p->B, c, cap)) {
+      ClusterSelArgs ca = {};
+      ca.vals = ts;
+      ca.stride = p->N;
+      ca.n = a.n;
+      ca.lo = a.lo;
+      ca.hi = a.hi;
+      ca.m = a.m;
+      ca.out = p->idx_out;
+      ca.out_stride = p->k;
+      ca.pooled_out = p->pooled_score_out;
+      ca.radius = radius;
+      ca.pool_mode = p->pool_mode;
+      g_last_path = REFORM_PATH_CLUSTER;
+      return launch_cluster_select<0>(ca, p->B, c, st);
+    }
   }
   a.out = p->idx_out;
   a.out_stride = p->k;
@@ -624,5 +686,6 @@ int reform_device_error(int clear) {
 }
 int reform_version(void) { return 100; }
 long long reform_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+int reform_debug_last_path(void) { return g_last_path; }
 
 }  // extern "C"

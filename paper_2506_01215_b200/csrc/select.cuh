@@ -158,8 +158,29 @@ __device__ __forceinline__ void sel_pass_params(int pass, int& shift, uint32_t& 
   else { shift = 0; digit_mask = 0x3FFu; prefix_mask = 0xFFFFFC00u; }
 }
 
-// Pools the raw token scores of one block's tile (Sec. 3.3).  tile: 2 * (kSelTile + 2 * radius)
-// floats of shared memory.  On return pooled_of(i) for the block's element i (0 <= i < kSelTile)
+// Bin walk over a shared-memory histogram of kSelBins bins from the top: the bin in which the
+// running count reaches `remaining`, and how many are still to take inside it.  All threads get
+// the same answer.  result: 2 uints of shared memory; scratch: 33.
+__device__ __forceinline__ void find_bin_shared(const uint32_t* hist, uint32_t remaining, uint32_t* scratch,
+                                                uint32_t* result, uint32_t& bin_out, uint32_t& rem_out) {
+  const int b0 = kSelBins - 1 - 2 * (int)threadIdx.x;
+  const uint32_t c0 = hist[b0], c1 = hist[b0 - 1];
+  uint32_t total;
+  const uint32_t before = block_excl_scan(c0 + c1, scratch, total);
+  if (threadIdx.x == 0) { result[0] = kSelBins - 1; result[1] = 0; }
+  __syncthreads();
+  if (before < remaining && remaining <= before + c0 + c1) {
+    if (remaining <= before + c0) { result[0] = b0; result[1] = remaining - before; }
+    else { result[0] = b0 - 1; result[1] = remaining - before - c0; }
+  }
+  __syncthreads();
+  bin_out = result[0];
+  rem_out = result[1];
+  __syncthreads();
+}
+
+// Pools the raw token scores of one block's tile (Sec. 3.3).  tile: 2 * (tile_len + 2 * radius)
+// floats of shared memory.  On return pooled_of(i) for the block's element i (0 <= i < tile_len)
 // is available through pool_result().  mode 0: maximum over the clipped window by log-step
 // doubling; mode 1: mean over the clipped window by direct summation in ascending token order.
 struct PoolTile {
@@ -170,9 +191,9 @@ struct PoolTile {
 };
 
 __device__ __forceinline__ PoolTile pool_prepare(float* tile, const float* __restrict__ src, long long base, int n,
-                                                 int radius, int mode) {
+                                                 int radius, int mode, int tile_len = kSelTile) {
   const int tid = threadIdx.x;
-  const int span = kSelTile + 2 * radius;
+  const int span = tile_len + 2 * radius;
   PoolTile p;
   p.radius = radius;
   p.window = 2 * radius + 1;
@@ -667,6 +688,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
                          int pool_mode = 0) {
   if (segs == 0) return REFORM_OK;
   if (!ts && a.n <= kSelBlockMaxN && segs >= kSelBlockMinSegs) {
+    g_last_path = REFORM_PATH_PER_SEGMENT;
     sel_block_kernel<<<segs, kSelThreads, 0, st>>>(a);
     count_launch();
     return check_launch();
@@ -677,6 +699,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
     if (ts) cudaFuncSetAttribute(sel_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int capacity = ts ? sel_fused_capacity<true>(smem) : sel_fused_capacity<false>(smem);
     if ((long long)a.blocks_per_seg * segs <= capacity) {
+      g_last_path = REFORM_PATH_COOPERATIVE;
       if (cudaMemsetAsync(ws_base, 0, L.zero_bytes, st) != cudaSuccess) return check_launch();
       SelFusedCtl* ctl = reinterpret_cast<SelFusedCtl*>(reinterpret_cast<char*>(ws_base) + L.ctl);
       void* args[] = {&a, &ctl, &ts, &pooled, &radius, &pool_mode, &dev_status};
@@ -691,6 +714,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
       return check_launch();
     }
   }
+  g_last_path = REFORM_PATH_PER_PASS;
   sel_init_kernel<<<segs, 256, 0, st>>>(a, segs);
   count_launch();
   if (ts) {

@@ -297,6 +297,102 @@ def test_evict_all_scores_equal_and_two_level_ties():
         assert torch.equal(kd.cpu(), ref["k"]) and torch.equal(sd.cpu().double(), ref["score"])
 
 
+def _score_kind(kind, shape, g):
+    if kind == "uniform":
+        return torch.rand(shape, generator=g)
+    if kind == "ties":                       # heavy ties, some negative, a -0.0
+        sc = (torch.rand(shape, generator=g) * 6).floor() / 4 - 0.5
+        sc[..., 5] = -0.0
+        return sc
+    if kind == "equal":                      # every candidate in one bin of every pass
+        return torch.full(shape, 0.37)
+    if kind == "lowbits":                    # agree in the leading 22 bits, differ in the last ones
+        return 1.0 + torch.randint(0, 50, shape, generator=g).float() * 2.0 ** -23
+    if kind == "heavy":                      # attention-mass-like: a few large values over a small floor
+        return torch.rand(shape, generator=g) ** 12 * 40 + torch.rand(shape, generator=g) * 1e-3
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("B,Hkv,d,n_keys,budget,sink,recent,dtype,kind", [
+    (4, 8, 64, 20480, 4096, 256, 256, torch.bfloat16, "uniform"),   # 32 clusters of 4 blocks
+    (4, 8, 16, 20001, 4097, 7, 9, torch.float32, "ties"),           # ragged lengths, odd capacity: scalar loads
+    (1, 12, 32, 40960, 8192, 256, 256, torch.bfloat16, "equal"),    # 12 clusters of 8
+    (3, 4, 8, 60000, 20000, 0, 0, torch.float32, "lowbits"),        # 12 clusters of 8, no forced rows
+    (3, 4, 8, 40963, 8192, 100, 3, torch.float32, "heavy"),
+    (4, 8, 8, 20480, 30000, 256, 256, torch.float32, "uniform"),    # under budget: nothing to choose
+    (4, 8, 8, 20480, 512, 256, 256, torch.float32, "uniform"),      # forced rows only
+])
+@pytest.mark.parametrize("in_place", [False, True])
+def test_evict_by_cluster_matches_oracle(B, Hkv, d, n_keys, budget, sink, recent, dtype, kind, in_place):
+    """Shapes that take the one-cluster-per-segment launch (checked through the path diagnostic):
+    selection through distributed shared memory, then the compaction by the same cluster, out of
+    place and in place, against the oracle's full sort bit for bit."""
+    g = torch.Generator().manual_seed(n_keys + budget)
+    cap = n_keys + (5 if n_keys % 2 else 8)
+    k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+    sc = _score_kind(kind, (B, Hkv, cap), g)
+    pos = torch.randint(0, 1 << 20, (B, Hkv, cap), generator=g, dtype=torch.int32)
+    cap_dst = cap if in_place else min(budget, n_keys) + 3
+    ref = oracle.evict_topk(k, v, sc, n_keys, budget, sink, recent, cap_dst=cap_dst, pos_src=pos)
+    ks, vs, ss, ps = k.to(DEV), v.to(DEV), sc.to(DEV), pos.to(DEV)
+    if in_place:
+        kd, vd, sd, pd = ks, vs, ss, ps
+    else:
+        kd = torch.zeros(B, Hkv, cap_dst, d, dtype=dtype, device=DEV)
+        vd, sd = torch.zeros_like(kd), torch.zeros(B, Hkv, cap_dst, device=DEV)
+        pd = torch.zeros(B, Hkv, cap_dst, dtype=torch.int32, device=DEV)
+    kept = torch.full((B, Hkv, budget), -1, dtype=torch.int32, device=DEV)
+    n_kept = R.evict_topk(ks, vs, ss, kd, vd, sd, n_keys, budget, sink, recent, pos_src=ps, pos_dst=pd,
+                          kept_idx=kept)
+    assert R.debug_last_path() == R.PATH_CLUSTER
+    torch.cuda.synchronize()
+    assert R.device_error() == 0
+    assert n_kept == ref["n_kept"]
+    assert torch.equal(kept.cpu()[:, :, :n_kept], ref["kept_idx"][:, :, :n_kept])
+    assert torch.equal(kd.cpu()[:, :, :n_kept].view(torch.uint8), ref["k"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(vd.cpu()[:, :, :n_kept].view(torch.uint8), ref["v"][:, :, :n_kept].view(torch.uint8))
+    assert torch.equal(sd.cpu()[:, :, :n_kept].double(), ref["score"][:, :, :n_kept])
+    assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept])
+    if in_place:
+        assert torch.equal(kd.cpu()[:, :, n_keys:], k[:, :, n_keys:])   # rows past the keys in use are untouched
+
+
+@pytest.mark.parametrize("B,N,E,nq,k,pool,keep,mode,quant", [
+    (1, 131072, 64, 4, 4096, 129, 256, "max", 0),     # the largest bank one cluster takes: 16 blocks
+    (2, 100003, 32, 3, 3000, 5, 0, "mean", 0),        # ragged, mean pooling
+    (3, 9000, 32, 2, 700, 1, 8, "max", 0),            # no pooling, clusters of 2
+    (1, 70001, 32, 2, 9000, 9, 100, "max", 8),        # quantised scores: heavy ties
+    (4, 65536, 32, 8, 60000, 129, 256, "max", 0),     # nearly everything selected
+])
+def test_retrieve_by_cluster_matches_oracle(B, N, E, nq, k, pool, keep, mode, quant):
+    """Banks of up to 131,072 tokens: pooling and selection by one cluster per sequence (checked
+    through the path diagnostic), against the oracle."""
+    g = torch.Generator().manual_seed(N + k)
+    bank = torch.randn(B, N, E, generator=g)
+    if quant:
+        bank = (bank * quant).round() / quant
+    bank = bank.bfloat16()
+    qs = torch.randn(B, nq, E, generator=g).bfloat16()
+    p = dict(scale=0.25, pool_window=pool, n_keep_head=keep, n_keep_tail=keep)
+    ref = oracle.retrieve_topk(bank, qs, N, k, pool_mode=mode, **p)
+    idx = torch.full((B, k), -1, dtype=torch.int32, device=DEV)
+    pooled = torch.zeros(B, N, device=DEV)
+    n_out = R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx, pooled_score_out=pooled,
+                            pool_mode=R.POOL_MEAN if mode == "mean" else R.POOL_MAX, **p)
+    assert R.debug_last_path() == R.PATH_CLUSTER
+    torch.cuda.synchronize()
+    assert n_out == ref["n_out"]
+    assert_scores_close(pooled, ref["pooled"], 1.0)
+    for b in range(B):
+        assert_index_sets_match(idx[b, :n_out].cpu(), ref["idx"][b], ref["pooled"][b])
+    # the same call without the optional pooled-score output selects the same tokens
+    idx2 = torch.full((B, k), -1, dtype=torch.int32, device=DEV)
+    R.retrieve_topk(bank.to(DEV), qs.to(DEV), N, k, idx2,
+                    pool_mode=R.POOL_MEAN if mode == "mean" else R.POOL_MAX, **p)
+    assert torch.equal(idx2, idx)
+
+
 def test_bounded_wait_runs_out_and_the_context_stays_usable():
     """Failure detection without a fault: the eviction's one-launch form is made to wait, for
     about a millisecond, on a flag that nothing sets.  Every block gives up, the kernel returns,
