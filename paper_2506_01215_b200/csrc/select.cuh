@@ -10,8 +10,7 @@
 // no atomics-dependent ordering anywhere and the result is bit-reproducible.
 //
 // The optional pooling (Sec. 3.3: max over the 2r+1 adjacent tokens) is fused
-// into the first histogram pass with a log-step sliding maximum in shared
-// memory.
+// into the first histogram pass: a grouped sliding maximum in shared memory.
 #pragma once
 
 #include "common.cuh"
@@ -179,62 +178,139 @@ __device__ __forceinline__ void find_bin_shared(const uint32_t* hist, uint32_t r
   __syncthreads();
 }
 
-// Pools the raw token scores of one block's tile (Sec. 3.3).  tile: 2 * (tile_len + 2 * radius)
-// floats of shared memory.  On return pooled_of(i) for the block's element i (0 <= i < tile_len)
-// is available through pool_result().  mode 0: maximum over the clipped window by log-step
-// doubling; mode 1: mean over the clipped window by direct summation in ascending token order.
+// Pools the raw token scores of one block's tile (Sec. 3.3).  tile: pool_tile_floats(tile_len,
+// radius) floats of shared memory, 16-byte aligned.  On return the pooled score of the block's
+// element i (0 <= i < tile_len, token base + i < n) is available through pool_result().
+//
+// mode 0, maximum over the clipped window [t - r, t + r]: the tile (with its halo of r on either
+// side, -inf outside the bank) is cut into aligned groups of eight; one pass leaves, per group, the
+// running maximum from its left end, the running maximum from its right end and the group's
+// maximum.  A window is then a suffix of its first group, a prefix of its last group and whole
+// groups in between: pooled = max(suffix[t - r], prefix[t + r], the groups strictly between).
+// One barrier, and r / 4 + 2 reads per element whatever the window.  Windows of fewer than nine
+// tokens are read directly.
+// mode 1, mean over the clipped window: direct summation in ascending token order.
+constexpr int kPoolGroup = 8;
+
+__host__ __device__ inline size_t pool_tile_floats(int tile_len, int radius) {
+  const size_t span8 = align_up((size_t)tile_len + 2 * (size_t)radius, kPoolGroup);
+  return 2 * span8 + span8 / kPoolGroup;
+}
+
 struct PoolTile {
-  float* cur;      // after pool_prepare: the array pool_result reads
-  int radius, window, len, mode;
-  long long base;  // first token of the block's tile
+  const float* x;     // mode 1 and short windows: the raw scores of the tile with its halo
+  const float* pre;   // grouped maximum: running maximum from the left end of each group
+  const float* suf;   //                  running maximum from the right end of each group
+  const float* grp;   //                  each group's maximum
+  int radius, mode;
+  bool grouped;
+  long long base;     // first token of the block's tile
   int n;
 };
 
 __device__ __forceinline__ PoolTile pool_prepare(float* tile, const float* __restrict__ src, long long base, int n,
                                                  int radius, int mode, int tile_len = kSelTile) {
   const int tid = threadIdx.x;
-  const int span = tile_len + 2 * radius;
+  const int span8 = (int)align_up((size_t)tile_len + 2 * (size_t)radius, kPoolGroup);
+  float* x = tile;
+  float* pre = tile + span8;
+  float* grp = tile + 2 * span8;
   PoolTile p;
   p.radius = radius;
-  p.window = 2 * radius + 1;
   p.mode = mode;
+  p.grouped = mode == 0 && radius >= kPoolGroup / 2;   // the window then always reaches into a second group
   p.base = base;
   p.n = n;
-  float* cur = tile;
-  float* nxt = tile + span;
-  for (int i = tid; i < span; i += kSelThreads) {
-    long long g = base - radius + i;
-    cur[i] = (g >= 0 && g < n) ? src[g] : -INFINITY;
-  }
-  __syncthreads();
-  int len = 1;
-  if (mode == 0) {
-    // W_p[j] = max cur[j .. j + 2^p - 1], doubling p while 2^(p+1) <= window
-    while (2 * len <= p.window) {
-      for (int i = tid; i < span; i += kSelThreads) {
-        float v = cur[i];
-        if (i + len < span) v = fmaxf(v, cur[i + len]);
-        nxt[i] = v;
-      }
-      __syncthreads();
-      float* t = cur; cur = nxt; nxt = t;
-      len *= 2;
+  p.x = x;
+  p.pre = pre;
+  p.suf = x;
+  p.grp = grp;
+  // eight independent loads per thread in flight at a time
+  for (int i0 = 0; i0 < span8; i0 += 8 * kSelThreads) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kSelThreads + tid;
+      const long long g = base - radius + i;
+      v[u] = (i < span8 && g >= 0 && g < n) ? __ldcg(src + g) : -INFINITY;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * kSelThreads + tid;
+      if (i < span8) x[i] = v[u];
     }
   }
-  p.cur = cur;
-  p.len = len;
+  __syncthreads();
+  if (p.grouped) {
+    for (int g = tid; g < span8 / kPoolGroup; g += kSelThreads) {
+      float4* xg = reinterpret_cast<float4*>(x + kPoolGroup * g);
+      const float4 a = xg[0], b = xg[1];
+      float4 pa, pb, sa, sb;
+      pa.x = a.x;                 pa.y = fmaxf(pa.x, a.y);  pa.z = fmaxf(pa.y, a.z);  pa.w = fmaxf(pa.z, a.w);
+      pb.x = fmaxf(pa.w, b.x);    pb.y = fmaxf(pb.x, b.y);  pb.z = fmaxf(pb.y, b.z);  pb.w = fmaxf(pb.z, b.w);
+      sb.w = b.w;                 sb.z = fmaxf(sb.w, b.z);  sb.y = fmaxf(sb.z, b.y);  sb.x = fmaxf(sb.y, b.x);
+      sa.w = fmaxf(sb.x, a.w);    sa.z = fmaxf(sa.w, a.z);  sa.y = fmaxf(sa.z, a.y);  sa.x = fmaxf(sa.y, a.x);
+      float4* pg = reinterpret_cast<float4*>(pre + kPoolGroup * g);
+      pg[0] = pa;
+      pg[1] = pb;
+      xg[0] = sa;   // the suffix maxima replace the group's raw scores (nobody else reads this group's x)
+      xg[1] = sb;
+      grp[g] = pb.w;
+    }
+    __syncthreads();
+  }
   return p;
 }
 
 // pooled score of the tile's element i (token base + i, which must be < n)
 __device__ __forceinline__ float pool_result(const PoolTile& p, int i) {
-  if (p.mode == 0) return fmaxf(p.cur[i], p.cur[i + p.window - p.len]);  // max(W[c], W[c + window - len])
+  if (p.mode == 0) {
+    const int L = i, R = i + 2 * p.radius;   // the window in tile coordinates (the tile starts r before its first element)
+    if (!p.grouped) {
+      float m = p.x[L];
+      for (int u = L + 1; u <= R; ++u) m = fmaxf(m, p.x[u]);
+      return m;
+    }
+    float m = fmaxf(p.suf[L], p.pre[R]);
+    for (int g = L / kPoolGroup + 1; g < R / kPoolGroup; ++g) m = fmaxf(m, p.grp[g]);
+    return m;
+  }
   const long long g = p.base + i;
   const int lo = (int)(g - p.radius < 0 ? -g : -p.radius);                  // offsets of the clipped window
   const int hi = (int)(g + p.radius > p.n - 1 ? p.n - 1 - g : p.radius);
   float sum = 0.f;
-  for (int u = lo; u <= hi; ++u) sum += p.cur[i + p.radius + u];
+  for (int u = lo; u <= hi; ++u) sum += p.x[i + p.radius + u];
   return sum / (float)(hi - lo + 1);
+}
+
+// The same for the eight consecutive elements i0 .. i0 + 7 (i0 a multiple of eight, every token
+// < n or its result unused): the eight windows start in one group and end in one or two, so the
+// whole groups they all cover are read once.
+__device__ __forceinline__ void pool_result8(const PoolTile& p, int i0, float (&out)[8]) {
+  if (!p.grouped) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out[j] = pool_result(p, i0 + j);
+    return;
+  }
+  const int gl = i0 / kPoolGroup;                       // first group of every window
+  const int q = (i0 + 2 * p.radius) / kPoolGroup;       // last group of window j: q, or q + 1 from j = 8 - rem on
+  const int rem = (i0 + 2 * p.radius) % kPoolGroup;
+  float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
+  int g = gl + 1;
+  for (; g + 3 < q; g += 4) {
+    c0 = fmaxf(c0, p.grp[g]);
+    c1 = fmaxf(c1, p.grp[g + 1]);
+    c2 = fmaxf(c2, p.grp[g + 2]);
+    c3 = fmaxf(c3, p.grp[g + 3]);
+  }
+  for (; g < q; ++g) c0 = fmaxf(c0, p.grp[g]);
+  const float core = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3));       // groups gl + 1 .. q - 1
+  const float core_q = q > gl ? fmaxf(core, p.grp[q]) : core;   // and group q, for the windows that end in q + 1
+  const float4 sa = *reinterpret_cast<const float4*>(p.suf + i0), sb = *reinterpret_cast<const float4*>(p.suf + i0 + 4);
+  const float sfx[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    out[j] = fmaxf(fmaxf(sfx[j], p.pre[i0 + 2 * p.radius + j]), rem + j < kPoolGroup ? core : core_q);
 }
 
 // One histogram pass.  POOL (pass 0 only): vals_in holds the raw token scores
@@ -244,7 +320,7 @@ template <bool POOL>
 __global__ void __launch_bounds__(kSelThreads)
 sel_hist_kernel(SelArgs a, int pass, const float* __restrict__ ts, float* __restrict__ pooled_out,
                 int radius, int pool_mode) {
-  extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
+  extern __shared__ __align__(16) float tile[];  // POOL: pool_tile_floats(kSelTile, radius) floats
   __shared__ uint32_t hist[kSelBins];
   __shared__ uint32_t scratch[33];
   __shared__ bool is_last;
@@ -444,11 +520,13 @@ __device__ __forceinline__ void sel_find_bin_local(const uint32_t* hist, uint32_
   __syncthreads();
 }
 
+// Two blocks per SM (32 registers per thread): the cooperative launch has to hold all blocks of the
+// call at once, 256 of them for a bank of 2^20 tokens.
 template <bool POOL>
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __launch_bounds__(kSelThreads, 2)
 sel_fused_kernel(SelArgs a, SelFusedCtl* ctl_all, const float* __restrict__ ts,
                  float* __restrict__ pooled_out, int radius, int pool_mode, int32_t* dev_status) {
-  extern __shared__ float tile[];  // POOL: 2 * (kSelTile + 2 * radius) floats
+  extern __shared__ __align__(16) float tile[];  // POOL: pool_tile_floats(kSelTile, radius) floats
   __shared__ uint32_t hist[kSelBins];
   __shared__ uint32_t scratch[33];
   __shared__ uint32_t result[2];
@@ -695,7 +773,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
   }
   dim3 grid(a.blocks_per_seg, segs);
   {
-    const size_t smem = ts ? sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius) : 0;
+    const size_t smem = ts ? sizeof(float) * pool_tile_floats(kSelTile, radius) : 0;
     if (ts) cudaFuncSetAttribute(sel_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     const int capacity = ts ? sel_fused_capacity<true>(smem) : sel_fused_capacity<false>(smem);
     if ((long long)a.blocks_per_seg * segs <= capacity) {
@@ -718,7 +796,7 @@ inline int launch_select(SelArgs a, int segs, const float* ts, float* pooled, in
   sel_init_kernel<<<segs, 256, 0, st>>>(a, segs);
   count_launch();
   if (ts) {
-    size_t smem = sizeof(float) * 2 * (kSelTile + 2 * (size_t)radius);
+    size_t smem = sizeof(float) * pool_tile_floats(kSelTile, radius);
     cudaFuncSetAttribute(sel_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     sel_hist_kernel<true><<<grid, kSelThreads, smem, st>>>(a, 0, ts, pooled, radius, pool_mode);
   } else {

@@ -57,10 +57,12 @@ struct ClusterSelSmem {
   uint2 cnt[kClMaxCluster];              // every block's (keys above the threshold, keys equal to it)
   uint32_t scratch[33];
   uint32_t result[2];
+  uint32_t pad[1];                       // the pooling tile that follows is read with 128-bit loads
 };
+static_assert(sizeof(ClusterSelSmem) % 16 == 0, "the pooling tile must start on a 16-byte boundary");
 
 inline size_t cluster_sel_smem_bytes(bool pool, int chunk, int radius) {
-  return sizeof(ClusterSelSmem) + (pool ? sizeof(float) * 2 * ((size_t)chunk + 2 * (size_t)radius) : 0);
+  return sizeof(ClusterSelSmem) + (pool ? sizeof(float) * pool_tile_floats(chunk, radius) : 0);
 }
 
 // MODE 0: pooling + selection (token selection).  MODE 1: selection + compaction (cache compression).
@@ -94,9 +96,7 @@ __global__ void __launch_bounds__(kSelThreads) cluster_select_kernel(const Clust
     if (POOL) {
       float* tile = reinterpret_cast<float*>(cl_smem_raw + sizeof(ClusterSelSmem));
       const PoolTile pt = pool_prepare(tile, src, base, a.n, a.radius, a.pool_mode, a.chunk);
-#pragma unroll
-      for (int j = 0; j < kClPer; ++j)
-        if (g0 + j < end) x[j] = pool_result(pt, kClPer * tid + j);
+      if (kClPer * tid < a.chunk) pool_result8(pt, kClPer * tid, x);   // elements past the bank's end are not used
       if (a.pooled_out) {
         float* dst = a.pooled_out + (long long)seg * a.stride;
         if ((a.stride & 3) == 0 && g0 + kClPer <= end) {
