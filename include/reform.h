@@ -173,11 +173,12 @@ int reform_chunk_step(const reform_chunk_params* p, reform_stream_t stream);
  * of them or none (a mixture, or any other overlap, is outside the contract;
  * equal pointers in a mixture are REFORM_ERR_INVALID_ARG).  The kept rows then
  * move down inside their own buffers and a layer needs one K/V buffer instead
- * of two.  In place needs rows of at most 256 bytes and a shape whose
- * selection blocks fit the device at once (segments up to 262,144 keys, about
- * a device's worth of 8,192-key blocks per call); otherwise the call returns
- * REFORM_ERR_UNSUPPORTED and nothing is launched.  The workspace needs no
- * clearing between calls.
+ * of two.  In place needs rows of at most 256 bytes and either segments of
+ * at most 131,072 keys (one thread-block cluster per segment, any number of
+ * segments) or a shape whose selection blocks fit the device at once (segments
+ * up to 262,144 keys, about a device's worth of 8,192-key blocks per call);
+ * otherwise the call returns REFORM_ERR_UNSUPPORTED and nothing is launched.
+ * The workspace needs no clearing between calls.
  * ------------------------------------------------------------------------ */
 typedef struct reform_evict_params {
   size_t struct_size;
@@ -238,11 +239,13 @@ int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t strea
 
 /* ------------------------------------------------------------------------
  * reform_debug_evict_wait_expiry -- diagnostic, no counterpart in the paper.
- * The kernels of this library never wait without a limit: a block that waits
+ * The kernels of this library never spin without a limit: a block that polls
  * for another block, for a copy or for the tensor cores gives up after a
  * bounded time, raises REFORM_DEV_TIMEOUT and lets the launch wind down with
- * the context intact.  This entry point lets a test see that happen without
- * faulting anything: it runs reform_evict_topk's one-launch form with the
+ * the context intact (the blocks of a thread-block cluster meet at the
+ * hardware's cluster barrier instead, which involves no polling loop).  This
+ * entry point lets a test see that happen without faulting anything: it runs
+ * reform_evict_topk's cooperative one-launch form with the
  * hand-off waits limited to wait_cycles SM clock cycles and with every
  * selection block waiting for one block more than the launch has -- a flag
  * that nothing ever sets.  Every block's first wait therefore runs out; the
@@ -250,7 +253,7 @@ int reform_evict_topk_static(const reform_evict_params* p, reform_stream_t strea
  * per-device error word, and the outputs are unspecified.  The call after it
  * behaves as if this one had not happened.
  * Arguments as for reform_evict_topk.  wait_cycles in (0, 400,000,000].
- * REFORM_ERR_UNSUPPORTED if the shape would not take the one-launch form
+ * REFORM_ERR_UNSUPPORTED if the shape cannot take that form
  * (nothing to choose, 48 or more short segments, more blocks than fit the
  * device at once).
  * ------------------------------------------------------------------------ */
