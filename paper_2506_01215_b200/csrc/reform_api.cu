@@ -323,7 +323,7 @@ static int evict_run(const reform_evict_params* p, cudaStream_t st, size_t need,
     // Taken in place always, and otherwise when the clusters run in one wave on enough blocks to
     // stream the kept rows at the device's rate (the cooperative form below spreads the copy over
     // the whole device whatever the number of segments).
-    const ClusterCapacity& cap = cluster_select_capacity<1>(cluster_sel_smem_bytes(false, 0, 0));
+    const ClusterCapacity cap = cluster_select_capacity<1>(cluster_sel_smem_bytes(false, 0, 0));
     const int c = cluster_select_size(segs, p->n_keys, cap);
     if (c && (in_place || (cluster_select_one_wave(segs, c, cap) && segs * c >= kClMinBlocksForCopy))) {
       ClusterSelArgs a = {};
@@ -595,7 +595,7 @@ int reform_retrieve_topk(const reform_retrieve_params* p, reform_stream_t stream
   {
     // banks of up to 16 x 8192 tokens: pooling and selection by one cluster per sequence
     const int radius = (p->pool_window - 1) / 2;
-    const ClusterCapacity& cap = cluster_select_capacity<0>(cluster_sel_smem_bytes(true, kClTile, radius));
+    const ClusterCapacity cap = cluster_select_capacity<0>(cluster_sel_smem_bytes(true, kClTile, radius));
     const int c = cluster_select_size(p->B, p->N, cap);
     if (c && cluster_select_one_wave(p->B, c, cap)) {
       ClusterSelArgs ca = {};

@@ -17,6 +17,8 @@
 
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "select.cuh"
 
@@ -262,13 +264,15 @@ struct ClusterCapacity {
 };
 
 template <int MODE>
-inline const ClusterCapacity& cluster_select_capacity(size_t smem) {
+inline ClusterCapacity cluster_select_capacity(size_t smem) {
   constexpr int kMaxDevices = 64;
   static ClusterCapacity cache[kMaxDevices] = {};
   static size_t cache_smem[kMaxDevices] = {0};
-  static const ClusterCapacity none = {};
+  static std::mutex guard;   // host threads may make their first call at the same time
+  const ClusterCapacity none = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return none;
+  std::lock_guard<std::mutex> lock(guard);
   if (cache_smem[dev] != 0 && smem <= cache_smem[dev]) return cache[dev];
   ClusterCapacity cap = {};
   const void* fn = (const void*)cluster_select_kernel<MODE>;
@@ -296,7 +300,7 @@ inline const ClusterCapacity& cluster_select_capacity(size_t smem) {
   }
   cache[dev] = cap;
   cache_smem[dev] = smem;
-  return cache[dev];
+  return cap;
 }
 
 // Cluster size for `segs` segments of n values: the smallest power of two whose blocks hold a
