@@ -934,6 +934,58 @@ def test_evict_seeded_random_shapes():
     assert R.device_error() == 0
 
 
+def test_evict_in_place_seeded_random_shapes():
+    """Fifty seeded shapes of the in-place cache compression (destinations == sources), which always
+    takes the one-cluster-per-segment launch: 1 to 12 segments of 1 to 131,072 keys (clusters of 1
+    to 16 blocks), capacities that allow and forbid vector key loads, all score distributions of
+    the out-of-place fuzz, each compared bit for bit with the oracle."""
+    import random
+    rnd = random.Random(20250603)
+    for case in range(50):
+        B = rnd.choice([1, 1, 2, 3]); Hkv = rnd.choice([1, 2, 4])
+        n = rnd.choice([1, 2, 9, 500, 4096, 8191, 8192, 8193, 16385, 30000, 40000, 65537, 100000, 131072])
+        if n > 50000:
+            B, Hkv = 1, rnd.choice([1, 2])
+        budget = max(1, min(n + rnd.choice([-1, 0, 5]), rnd.choice([1, 8, 100, n // 5 + 1, n // 2 + 1, n - 1, n])))
+        sink = rnd.choice([0, 0, 1, 4, budget // 3])
+        recent = rnd.choice([0, 0, 1, 4, budget // 3])
+        if sink + recent > budget or sink + recent > n:
+            sink, recent = 0, min(recent, budget, n) // 2
+        cap = n + rnd.choice([0, 1, 3, 4, 8])
+        d = rnd.choice([4, 8, 64])
+        dtype = rnd.choice([torch.float32, torch.bfloat16]) if d >= 8 else torch.float32
+        g = torch.Generator().manual_seed(case * 7919 + 11)
+        k = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+        v = torch.randn(B, Hkv, cap, d, generator=g).to(dtype)
+        kind = rnd.choice(["uniform", "heavy_tail", "tied", "two_level", "constant", "signed"])
+        u = torch.rand(B, Hkv, cap, generator=g)
+        sc = {"uniform": u, "heavy_tail": torch.exp(8 * u) / 2981.0, "tied": (u * 7).floor() / 7,
+              "two_level": 1.0 + (u * 40).floor() * 2.0 ** -23, "constant": torch.full_like(u, 0.25),
+              "signed": (u - 0.5) * 3}[kind]
+        with_pos, with_kept = rnd.random() < 0.5, rnd.random() < 0.7
+        pos = torch.randint(0, 1 << 20, (B, Hkv, cap), generator=g, dtype=torch.int32) if with_pos else None
+        ref = oracle.evict_topk(k, v, sc, n, budget, sink, recent, cap_dst=cap, pos_src=pos)
+        kd, vd, sd = k.to(DEV), v.to(DEV), sc.to(DEV)
+        pd = pos.to(DEV) if with_pos else None
+        kept = torch.full((B, Hkv, budget), -1, dtype=torch.int32, device=DEV) if with_kept else None
+        status = "case %d: B %d Hkv %d n %d budget %d sink %d recent %d cap %d d %d %s" % (
+            case, B, Hkv, n, budget, sink, recent, cap, d, kind)
+        n_kept = R.evict_topk(kd, vd, sd, kd, vd, sd, n, budget, sink, recent, pos_src=pd, pos_dst=pd,
+                              kept_idx=kept)
+        assert R.debug_last_path() == R.PATH_CLUSTER, status
+        torch.cuda.synchronize()
+        assert n_kept == ref["n_kept"], status
+        if with_kept:
+            assert torch.equal(kept.cpu()[:, :, :n_kept], ref["kept_idx"][:, :, :n_kept]), status
+        assert torch.equal(kd.cpu()[:, :, :n_kept].view(torch.uint8), ref["k"][:, :, :n_kept].view(torch.uint8)), status
+        assert torch.equal(vd.cpu()[:, :, :n_kept].view(torch.uint8), ref["v"][:, :, :n_kept].view(torch.uint8)), status
+        assert torch.equal(sd.cpu()[:, :, :n_kept].double(), ref["score"][:, :, :n_kept]), status
+        if with_pos:
+            assert torch.equal(pd.cpu()[:, :, :n_kept], ref["pos"][:, :, :n_kept]), status
+        assert torch.equal(kd.cpu()[:, :, n:], k[:, :, n:]), status
+    assert R.device_error() == 0
+
+
 def test_retrieve_seeded_random_shapes():
     """Forty seeded shapes of the retrieval (bank lengths on and off the tile grids, 1 to 64 queries,
     row widths that take the tensor-core scan and ones that do not, fp32 and bf16, pooling windows 1
