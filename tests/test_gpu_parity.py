@@ -934,6 +934,59 @@ def test_evict_seeded_random_shapes():
     assert R.device_error() == 0
 
 
+def test_two_host_threads_on_their_own_streams():
+    """The library's per-process state (launch-form caches, epochs, counters) under two host
+    threads that call it at the same time, each on its own stream with its own buffers and
+    workspaces: thirty rounds of cache compression (cooperative and cluster forms) and token
+    selection per thread, every result equal to the oracle's."""
+    import threading
+    g = torch.Generator().manual_seed(31)
+    cases = []
+    for n, budget, B, Hkv in ((9000, 2048, 1, 4), (20480, 4096, 4, 8)):
+        k = torch.randn(B, Hkv, n, 8, generator=g)
+        sc = torch.rand(B, Hkv, n, generator=g)
+        cases.append((k, sc, n, budget, oracle.evict_topk(k, k, sc, n, budget, 16, 16, cap_dst=budget)))
+    N, E, kk = 20000, 32, 1500
+    bank = torch.randn(1, N, E, generator=g).bfloat16()
+    qs = torch.randn(1, 3, E, generator=g).bfloat16()
+    rp = dict(scale=0.25, pool_window=9, n_keep_head=4, n_keep_tail=4)
+    rref = oracle.retrieve_topk(bank, qs, N, kk, **rp)
+    errors = []
+
+    def worker(tid):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                dev = [(k.to(DEV), sc.to(DEV)) for k, sc, _, _, _ in cases]
+                bank_d, qs_d = bank.to(DEV), qs.to(DEV)
+                ws = torch.empty(64 << 20, dtype=torch.uint8, device=DEV)
+                for it in range(30):
+                    for (k, sc, n, budget, ref), (kd_src, sc_d) in zip(cases, dev):
+                        B, Hkv = k.shape[:2]
+                        kd = torch.zeros(B, Hkv, budget, 8, device=DEV)
+                        vd, sd = torch.zeros_like(kd), torch.zeros(B, Hkv, budget, device=DEV)
+                        kept = torch.zeros(B, Hkv, budget, dtype=torch.int32, device=DEV)
+                        R.evict_topk(kd_src, kd_src, sc_d, kd, vd, sd, n, budget, 16, 16, kept_idx=kept, ws=ws,
+                                     stream=st)
+                        st.synchronize()
+                        assert torch.equal(kept.cpu(), ref["kept_idx"]), (tid, it, n)
+                        assert torch.equal(kd.cpu(), ref["k"]), (tid, it, n)
+                    idx = torch.full((1, kk), -1, dtype=torch.int32, device=DEV)
+                    R.retrieve_topk(bank_d, qs_d, N, kk, idx, ws=ws, stream=st, **rp)
+                    st.synchronize()
+                    assert_index_sets_match(idx[0].cpu(), rref["idx"][0], rref["pooled"][0])
+        except Exception as e:   # reported by the main thread
+            errors.append((tid, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert R.device_error() == 0
+
+
 def test_evict_in_place_seeded_random_shapes():
     """Fifty seeded shapes of the in-place cache compression (destinations == sources), which always
     takes the one-cluster-per-segment launch: 1 to 12 segments of 1 to 131,072 keys (clusters of 1
