@@ -39,6 +39,7 @@ scan_sm100_kernel(const __grid_constant__ CUtensorMap tmBank, const __grid_const
                   float* __restrict__ ts, long long N, int E, int nq, int n_pad, int n_stages, float scale,
                   int tiles_per_seq, int32_t* dev_status) {
   extern __shared__ uint8_t smem_raw[];
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent selection may be placed as SMs free up
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int KB = E / 64;
   const uint32_t q_box_bytes = (uint32_t)n_pad * 128;

@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kSelThreads) cluster_select_kernel(const Clust
 #pragma unroll
     for (int j = 0; j < kClPer; ++j) x[j] = 0.f;
     if (POOL) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // the scan's scores are complete from here on
       float* tile = reinterpret_cast<float*>(cl_smem_raw + sizeof(ClusterSelSmem));
       const PoolTile pt = pool_prepare(tile, src, base, a.n, a.radius, a.pool_mode, a.chunk);
       if (kClPer * tid < a.chunk) pool_result8(pt, kClPer * tid, x);   // elements past the bank's end are not used
@@ -331,13 +332,17 @@ inline int launch_cluster_select(ClusterSelArgs a, int segs, int c, cudaStream_t
   cfg.blockDim = dim3(kSelThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = c;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // token selection: placed while the scan that writes its scores drains (the kernel waits for the
+  // scan's completion before its first read of them)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = MODE == 0 ? 2 : 1;
   cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_select_kernel<MODE>, a);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
